@@ -1,0 +1,158 @@
+"""CPU oracle (test infrastructure only).
+
+Thin numpy/ctypes wrapper over ``oracle.c``: plain, slow, one-row-at-a-time
+definitions of causal grouped-query attention (Sec. 3.2 of the paper) and of
+the token log-probability (Sec. 3.1).  Only the tests, the smoke check and
+the benchmark's CPU-baseline leg may import this package; it imports nothing
+from the CUDA package and the CUDA package never imports it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liboracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile oracle.c with gcc (OpenMP) into liboracle.so next to it."""
+    srcs = [os.path.join(_HERE, "oracle.c"), os.path.join(_HERE, "oracle_impl.inc")]
+    if not force and os.path.exists(_LIB_PATH):
+        if all(os.path.getmtime(_LIB_PATH) >= os.path.getmtime(s) for s in srcs):
+            return _LIB_PATH
+    cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99", srcs[0], "-o", _LIB_PATH, "-lm"]
+    subprocess.run(cmd, check=True, cwd=_HERE)
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB_PATH)
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _i64(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int64))
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
+
+
+def _real(f32: bool):
+    return (np.float32, "_f32") if f32 else (np.float64, "")
+
+
+def attn_packed(q, k, v, cu_seqlens, scale: float, f32: bool = False):
+    """q [tot,Hq,d], k/v [tot,Hkv,d] -> (out [tot,Hq,d], lse [tot,Hq])."""
+    q, k, v, cu = _f32(q), _f32(k), _f32(v), _i32(cu_seqlens)
+    tot, Hq, d = q.shape
+    Hkv = k.shape[1]
+    assert k.shape == (tot, Hkv, d) and v.shape == k.shape and cu[-1] == tot
+    dt, sfx = _real(f32)
+    out = np.empty((tot, Hq, d), dtype=dt)
+    lse = np.empty((tot, Hq), dtype=dt)
+    rc = getattr(lib(), "oracle_attn_packed" + sfx)(
+        _p(q), _p(k), _p(v), _p(cu), ctypes.c_int(len(cu) - 1), ctypes.c_int(Hq),
+        ctypes.c_int(Hkv), ctypes.c_int(d), ctypes.c_double(scale), _p(out), _p(lse))
+    assert rc == 0
+    return out, lse
+
+
+def attn_paged(q, cu_seqlens_q, ctx_lens, k_cache, v_cache, block_table, scale: float,
+               f32: bool = False):
+    """q [totq,Hq,d]; caches [num_pages,Hkv,page,d]; block_table [S,max_blocks]."""
+    q, kc, vc = _f32(q), _f32(k_cache), _f32(v_cache)
+    cu, ctx, bt = _i32(cu_seqlens_q), _i32(ctx_lens), _i32(block_table)
+    totq, Hq, d = q.shape
+    _, Hkv, page, d2 = kc.shape
+    assert d2 == d and vc.shape == kc.shape and bt.ndim == 2 and bt.shape[0] == len(ctx)
+    dt, sfx = _real(f32)
+    out = np.empty((totq, Hq, d), dtype=dt)
+    lse = np.empty((totq, Hq), dtype=dt)
+    rc = getattr(lib(), "oracle_attn_paged" + sfx)(
+        _p(q), _p(cu), _p(ctx), _p(kc), _p(vc), _p(bt), ctypes.c_int(bt.shape[1]),
+        ctypes.c_int(len(ctx)), ctypes.c_int(Hq), ctypes.c_int(Hkv), ctypes.c_int(d),
+        ctypes.c_int(page), ctypes.c_double(scale), _p(out), _p(lse))
+    assert rc == 0
+    return out, lse
+
+
+def attn_rows(q_rows, k, v, kv_off, kv_len, scale: float, f32: bool = False):
+    """Row r: query q_rows[r] against k/v[kv_off[r] : kv_off[r]+kv_len[r]] (flat [totk,d])."""
+    q_rows, k, v = _f32(q_rows), _f32(k), _f32(v)
+    off, ln = _i64(kv_off), _i64(kv_len)
+    n, d = q_rows.shape
+    assert k.shape[1] == d and v.shape == k.shape
+    assert n == 0 or int((off + ln).max()) <= k.shape[0]
+    dt, sfx = _real(f32)
+    out = np.empty((n, d), dtype=dt)
+    lse = np.empty((n,), dtype=dt)
+    rc = getattr(lib(), "oracle_attn_rows" + sfx)(
+        _p(q_rows), _p(k), _p(v), _p(off), _p(ln), ctypes.c_int64(n), ctypes.c_int(d),
+        ctypes.c_double(scale), _p(out), _p(lse))
+    assert rc == 0
+    return out, lse
+
+
+def attn_probs(q_row, k, v, scale: float, f32: bool = False):
+    """Normalised attention weights and output of one row over all rows of k/v [n,d]."""
+    q_row, k, v = _f32(q_row), _f32(k), _f32(v)
+    n, d = k.shape
+    dt, sfx = _real(f32)
+    probs = np.empty((n,), dtype=dt)
+    out = np.empty((d,), dtype=dt)
+    rc = getattr(lib(), "oracle_attn_probs" + sfx)(
+        _p(q_row), _p(k), _p(v), ctypes.c_int64(n), ctypes.c_int(d), ctypes.c_double(scale),
+        _p(probs), _p(out))
+    assert rc == 0
+    return probs, out
+
+
+def token_logprob(hidden, W, target, inv_temperature: float = 1.0, f32: bool = False):
+    """hidden [T,H], W [V,H], target [T] -> (logprob [T], lse [T])."""
+    hidden, W, target = _f32(hidden), _f32(W), _i32(target)
+    T, H = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == H and target.shape == (T,)
+    dt, sfx = _real(f32)
+    lp = np.empty((T,), dtype=dt)
+    lse = np.empty((T,), dtype=dt)
+    rc = getattr(lib(), "oracle_token_logprob" + sfx)(
+        _p(hidden), _p(W), _p(target), ctypes.c_int64(T), ctypes.c_int(H), ctypes.c_int(V),
+        ctypes.c_double(inv_temperature), _p(lp), _p(lse))
+    assert rc == 0
+    return lp, lse
+
+
+def log_softmax_row(hidden_row, W, inv_temperature: float = 1.0, f32: bool = False):
+    """The full log-softmax row [V] of one token."""
+    hidden_row, W = _f32(hidden_row), _f32(W)
+    V, H = W.shape
+    dt, sfx = _real(f32)
+    out = np.empty((V,), dtype=dt)
+    rc = getattr(lib(), "oracle_log_softmax_row" + sfx)(
+        _p(hidden_row), _p(W), ctypes.c_int(H), ctypes.c_int(V),
+        ctypes.c_double(inv_temperature), _p(out))
+    assert rc == 0
+    return out
