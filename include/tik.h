@@ -1,0 +1,139 @@
+/* tik: bitwise-consistent causal GQA attention and token log-probability for B200 (sm_100a).
+ *
+ * C ABI.  Unless stated otherwise every data pointer is a DEVICE pointer owned by the
+ * caller; the library borrows it until the work queued on `stream` (a cudaStream_t
+ * passed as void*) has completed.  Calls are asynchronous, never synchronise and never
+ * read device memory on the host.  After tik_create the library allocates no device
+ * memory: scratch comes from the caller (`ws`, sized by tik_workspace_bytes).
+ *
+ * Layouts (bf16 unless noted, all contiguous):
+ *   packed tokens    [tokens][heads][d]
+ *   KV cache         [num_pages][Hkv][page_size][d], separate K and V pools.  Rows of a
+ *                    page that lie beyond a sequence's context must hold finite values
+ *                    (zero-initialise the pool): they are multiplied by weight 0.
+ *   block table      int32 [S][max_blocks]: physical page of each logical page.
+ *   cu_seqlens       int32 [S+1] exclusive prefix sums of per-sequence token counts.
+ *
+ * The promise (paper Sec. 4.1, Eq. 1; Sec. 3.2 "same query data and causal KV prefix"):
+ * for a fixed tik_contract_id(), the output bits of an attention row depend only on that
+ * row's query, the values of its causal K/V prefix, softmax_scale and d -- not on the
+ * entry point (train forward, prefill, decode), batch size or slot, packing order, page
+ * size or placement, grid size or stream.  Likewise a log-probability depends only on
+ * its hidden row, lm_head, target and inv_temperature, not on T or the row's index.
+ *
+ * Supported domain: d in {64,128}; page_size in {16,32,64,128}; Hq % Hkv == 0 and
+ * Hq/Hkv <= 32; H % 64 == 0; all base pointers 16-byte aligned.  Anything else returns
+ * TIK_ERR_UNSUPPORTED.  Nothing traps or aborts.
+ */
+#ifndef TIK_H
+#define TIK_H
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tik_ctx tik_ctx;   /* opaque, per device */
+typedef int tik_status;
+
+#define TIK_OK 0
+#define TIK_ERR_INVALID_ARG (-1)   /* null pointer, negative size, Hq % Hkv != 0, bad scale */
+#define TIK_ERR_UNSUPPORTED (-2)   /* outside the supported domain above */
+#define TIK_ERR_WORKSPACE (-3)     /* ws_bytes smaller than tik_workspace_bytes(...) */
+#define TIK_ERR_CUDA (-4)          /* a CUDA call failed; text via tik_last_error */
+
+/* device-side flags reported by tik_device_status */
+#define TIK_DEV_BAD_BLOCK 1        /* block-table entry outside [0,num_pages): page read as zeros */
+#define TIK_DEV_BAD_TARGET 2       /* target id outside [0,V): logprob = NaN */
+#define TIK_DEV_WAIT_EXPIRED 4     /* an in-kernel bounded wait ran out (outputs invalid) */
+
+#define TIK_OP_ATTN_TRAIN_FWD 0
+#define TIK_OP_ATTN_PREFILL 1
+#define TIK_OP_ATTN_DECODE 2
+#define TIK_OP_TOKEN_LOGPROB 3
+
+/* Create / destroy the per-device context (host memory plus one small device status
+ * word).  `device` is a CUDA ordinal.  tik_create is the only call that allocates. */
+tik_status tik_create(tik_ctx** out, int device);
+tik_status tik_destroy(tik_ctx* ctx);
+
+const char* tik_status_str(tik_status s);
+/* Text of the last TIK_ERR_CUDA / argument error of this context (host string). */
+const char* tik_last_error(const tik_ctx* ctx);
+/* Identifies the numerical contract (tile sizes, MMA shape, exp variant, sum shape).
+ * Outputs are bit-comparable only between builds with the same id. */
+const char* tik_contract_id(void);
+
+/* Scratch bytes an operator needs.  rows_or_batch: decode batch B, or log-prob rows T;
+ * ignored (0) for train forward / prefill, which need none.  max_ctx: largest context
+ * length (decode).  H, V only for the log-prob op.  Returns 0 when no scratch is needed. */
+size_t tik_workspace_bytes(int op, int64_t rows_or_batch, int Hq, int Hkv, int d,
+                           int64_t max_ctx, int H, int V);
+
+/* Synchronises `stream`, then reads and clears the device flags (TIK_DEV_*). */
+tik_status tik_device_status(tik_ctx* ctx, void* stream, int* out_flags);
+
+/* Policy-update forward attention over packed variable-length sequences (paper Sec. 4.1:
+ * the full-sequence entry point applied to prompt||response).  Token t of a sequence
+ * attends keys 0..t of the same sequence; query head h uses KV head h / (Hq/Hkv).
+ *   q [total_tokens][Hq][d], k, v [total_tokens][Hkv][d]  -> o [total_tokens][Hq][d]
+ *   lse: optional fp32 [total_tokens][Hq] (natural-log log-sum-exp of the scaled scores)
+ *   cu_seqlens: device int32 [S+1]; max_seqlen: host upper bound on any sequence length
+ *   (sizes the grid; may be larger than the true maximum). */
+tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const void* v, void* o,
+                              float* lse, const int32_t* cu_seqlens, int S,
+                              int64_t total_tokens, int max_seqlen, int Hq, int Hkv, int d,
+                              float softmax_scale, void* stream);
+
+/* Indexed KV-cache write (paper Sec. 4.1: a rollout-only operator; exact copy).  The new
+ * tokens of sequence s are rows cu_seqlens_new[s] .. cu_seqlens_new[s+1]-1 of k_new/v_new
+ * ([total_new][Hkv][d]) and land at positions ctx_lens[s]-n_s .. ctx_lens[s]-1, where
+ * ctx_lens[s] is the context length AFTER the write.  Position p goes to page
+ * block_table[s][p / page_size], row p % page_size. */
+tik_status tik_kv_cache_write(tik_ctx* ctx, const void* k_new, const void* v_new,
+                              const int32_t* cu_seqlens_new, const int32_t* ctx_lens,
+                              void* k_cache, void* v_cache, const int32_t* block_table,
+                              int max_blocks, int S, int64_t total_new, int Hkv, int d,
+                              int page_size, int num_pages, void* stream);
+
+/* Rollout prefill attention (paper Sec. 4.1: the full-sequence entry point applied to a
+ * prompt) against the paged cache, which must already hold the keys/values of positions
+ * 0 .. ctx_lens[s]-1 (tik_kv_cache_write first).  Query i of sequence s sits at absolute
+ * position ctx_lens[s] - q_len[s] + i and attends keys 0..position, so a cached prefix
+ * (chunked prefill) is supported.  max_q_len / max_ctx_len: host upper bounds. */
+tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse,
+                            const int32_t* cu_seqlens_q, const int32_t* ctx_lens,
+                            const void* k_cache, const void* v_cache,
+                            const int32_t* block_table, int max_blocks, int S, int64_t total_q,
+                            int max_q_len, int max_ctx_len, int Hq, int Hkv, int d,
+                            int page_size, int num_pages, float softmax_scale, void* stream);
+
+/* Token-wise decode attention (paper Sec. 4.1: the decode entry point): one query token
+ * per sequence at position ctx_lens[b]-1 (its own key/value already written) against keys
+ * 0..ctx_lens[b]-1.  q, o [B][Hq][d]; lse optional fp32 [B][Hq].  A slot with
+ * ctx_lens[b] <= 0 is skipped and its output rows are left untouched.  The KV range is
+ * split into fixed 2048-key chunks whose partial results go through `ws` and are folded in
+ * ascending order by a second kernel on the same stream (fixed-order split-KV combine). */
+tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse,
+                           const int32_t* ctx_lens, const void* k_cache, const void* v_cache,
+                           const int32_t* block_table, int max_blocks, int B, int max_ctx_len,
+                           int Hq, int Hkv, int d, int page_size, int num_pages,
+                           float softmax_scale, void* ws, size_t ws_bytes, void* stream);
+
+/* Token log-probabilities (paper Sec. 3.1): z = inv_temperature * hidden[t] . lm_head[v]
+ * for all v in fp32 (never rounded to bf16), logprob[t] = z[target[t]] - logsumexp_v z.
+ *   hidden [T][H], lm_head [V][H] (row v = class v), target_ids int32 [T]
+ *   -> logprob fp32 [T]; lse optional fp32 [T].
+ * The logits are never materialised: the GEMM runs on tensor cores with a fixed
+ * ascending-K accumulation and is fused with a chunked log-sum-exp whose partial results
+ * (per 1024-column super-chunk) go through `ws` and are folded in ascending order. */
+tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_head,
+                             const int32_t* target_ids, float* logprob, float* lse, int64_t T,
+                             int H, int V, float inv_temperature, void* ws, size_t ws_bytes,
+                             void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TIK_H */

@@ -1,0 +1,208 @@
+"""ctypes binding of libtik.so: argument marshalling only.
+
+Every function takes torch CUDA tensors (device memory and the current
+stream come from torch), checks dtypes/contiguity, and forwards raw pointers
+and sizes to the C entry point of the same name.  All arithmetic happens in
+the library's kernels; there is no fallback, and a missing library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+OK = 0
+OP_ATTN_TRAIN_FWD, OP_ATTN_PREFILL, OP_ATTN_DECODE, OP_TOKEN_LOGPROB = 0, 1, 2, 3
+DEV_BAD_BLOCK, DEV_BAD_TARGET, DEV_WAIT_EXPIRED = 1, 2, 4
+
+_lib = None
+_ctx = {}
+
+
+class TikError(RuntimeError):
+    pass
+
+
+def load(build_if_missing: bool = False) -> ctypes.CDLL:
+    """Loads libtik.so (optionally building it first).  Raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if build_if_missing:
+        _build.build()
+    if not os.path.exists(path):
+        raise TikError("libtik.so is not built (%s); run `python -m paper_2609_35140_b200.build`. "
+                       "There is no fallback path." % path)
+    lib = ctypes.CDLL(path)
+    c = ctypes
+    vp, i32, i64, f32, sz = c.c_void_p, c.c_int, c.c_int64, c.c_float, c.c_size_t
+    lib.tik_create.argtypes = [c.POINTER(vp), i32]
+    lib.tik_destroy.argtypes = [vp]
+    lib.tik_status_str.argtypes = [i32]
+    lib.tik_status_str.restype = c.c_char_p
+    lib.tik_last_error.argtypes = [vp]
+    lib.tik_last_error.restype = c.c_char_p
+    lib.tik_contract_id.restype = c.c_char_p
+    lib.tik_workspace_bytes.argtypes = [i32, i64, i32, i32, i32, i64, i32, i32]
+    lib.tik_workspace_bytes.restype = sz
+    lib.tik_device_status.argtypes = [vp, vp, c.POINTER(i32)]
+    lib.tik_attn_train_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, vp]
+    lib.tik_kv_cache_write.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, i32, i32, vp]
+    lib.tik_attn_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, i32, i32,
+                                     i32, i32, i32, f32, vp]
+    lib.tik_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32,
+                                    f32, vp, sz, vp]
+    lib.tik_token_logprob.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, f32, vp, sz, vp]
+    for name in ("tik_create", "tik_destroy", "tik_device_status", "tik_attn_train_fwd",
+                 "tik_kv_cache_write", "tik_attn_prefill", "tik_attn_decode", "tik_token_logprob"):
+        getattr(lib, name).restype = i32
+    _lib = lib
+    return lib
+
+
+def contract_id() -> str:
+    return load().tik_contract_id().decode()
+
+
+def context(device: Optional[int] = None) -> ctypes.c_void_p:
+    """The per-device library context (created on first use)."""
+    lib = load()
+    if not torch.cuda.is_available():
+        raise TikError("tik needs a CUDA device; there is no CPU path")
+    dev = torch.cuda.current_device() if device is None else device
+    if dev not in _ctx:
+        h = ctypes.c_void_p()
+        rc = lib.tik_create(ctypes.byref(h), dev)
+        if rc != OK:
+            raise TikError("tik_create failed: %s" % lib.tik_status_str(rc).decode())
+        _ctx[dev] = h
+    return _ctx[dev]
+
+
+def _check(rc: int, ctx) -> None:
+    if rc != OK:
+        lib = load()
+        raise TikError("%s: %s" % (lib.tik_status_str(rc).decode(), lib.tik_last_error(ctx).decode()))
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise TikError("tensors must be contiguous CUDA tensors")
+    if dtype is not None and t.dtype != dtype:
+        raise TikError("expected dtype %s, got %s" % (dtype, t.dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def workspace_bytes(op: int, rows_or_batch: int = 0, Hq: int = 0, Hkv: int = 0, d: int = 0,
+                    max_ctx: int = 0, H: int = 0, V: int = 0) -> int:
+    return int(load().tik_workspace_bytes(op, rows_or_batch, Hq, Hkv, d, max_ctx, H, V))
+
+
+def device_status() -> int:
+    """Synchronises the current stream; returns and clears the device flags."""
+    ctx = context()
+    flags = ctypes.c_int(0)
+    _check(load().tik_device_status(ctx, _stream(), ctypes.byref(flags)), ctx)
+    return flags.value
+
+
+def tik_attn_train_fwd(q, k, v, cu_seqlens, max_seqlen: int, softmax_scale: float,
+                       o: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
+    """q [tot,Hq,d], k/v [tot,Hkv,d] bf16, cu_seqlens int32 [S+1] (device) -> o [tot,Hq,d]."""
+    ctx = context()
+    tot, Hq, d = q.shape
+    Hkv = k.shape[1]
+    if o is None:
+        o = torch.empty_like(q)
+    bf = torch.bfloat16
+    rc = load().tik_attn_train_fwd(ctx, _ptr(q, bf), _ptr(k, bf), _ptr(v, bf), _ptr(o, bf),
+                                   _ptr(lse, torch.float32), _ptr(cu_seqlens, torch.int32),
+                                   cu_seqlens.numel() - 1, tot, max_seqlen, Hq, Hkv, d,
+                                   softmax_scale, _stream())
+    _check(rc, ctx)
+    return o
+
+
+def tik_kv_cache_write(k_new, v_new, cu_seqlens_new, ctx_lens, k_cache, v_cache, block_table):
+    """Copies new K/V rows into the paged caches [num_pages,Hkv,page,d] in place."""
+    ctx = context()
+    bf = torch.bfloat16
+    num_pages, Hkv, page, d = k_cache.shape
+    rc = load().tik_kv_cache_write(ctx, _ptr(k_new, bf), _ptr(v_new, bf),
+                                   _ptr(cu_seqlens_new, torch.int32), _ptr(ctx_lens, torch.int32),
+                                   _ptr(k_cache, bf), _ptr(v_cache, bf),
+                                   _ptr(block_table, torch.int32), block_table.shape[1],
+                                   ctx_lens.numel(), k_new.shape[0], Hkv, d, page, num_pages, _stream())
+    _check(rc, ctx)
+
+
+def tik_attn_prefill(q, cu_seqlens_q, ctx_lens, k_cache, v_cache, block_table, max_q_len: int,
+                     max_ctx_len: int, softmax_scale: float, o: Optional[torch.Tensor] = None,
+                     lse: Optional[torch.Tensor] = None):
+    """q [totq,Hq,d] against the paged cache -> o [totq,Hq,d]."""
+    ctx = context()
+    bf = torch.bfloat16
+    totq, Hq, d = q.shape
+    num_pages, Hkv, page, _ = k_cache.shape
+    if o is None:
+        o = torch.empty_like(q)
+    rc = load().tik_attn_prefill(ctx, _ptr(q, bf), _ptr(o, bf), _ptr(lse, torch.float32),
+                                 _ptr(cu_seqlens_q, torch.int32), _ptr(ctx_lens, torch.int32),
+                                 _ptr(k_cache, bf), _ptr(v_cache, bf), _ptr(block_table, torch.int32),
+                                 block_table.shape[1], ctx_lens.numel(), totq, max_q_len, max_ctx_len,
+                                 Hq, Hkv, d, page, num_pages, softmax_scale, _stream())
+    _check(rc, ctx)
+    return o
+
+
+def tik_attn_decode(q, ctx_lens, k_cache, v_cache, block_table, max_ctx_len: int, softmax_scale: float,
+                    ws: Optional[torch.Tensor] = None, o: Optional[torch.Tensor] = None,
+                    lse: Optional[torch.Tensor] = None):
+    """q [B,Hq,d]: one token per sequence against the paged cache -> o [B,Hq,d]."""
+    ctx = context()
+    bf = torch.bfloat16
+    B, Hq, d = q.shape
+    num_pages, Hkv, page, _ = k_cache.shape
+    need = workspace_bytes(OP_ATTN_DECODE, B, Hq, Hkv, d, max_ctx_len)
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+    if o is None:
+        o = torch.empty_like(q)
+    rc = load().tik_attn_decode(ctx, _ptr(q, bf), _ptr(o, bf), _ptr(lse, torch.float32),
+                                _ptr(ctx_lens, torch.int32), _ptr(k_cache, bf), _ptr(v_cache, bf),
+                                _ptr(block_table, torch.int32), block_table.shape[1], B, max_ctx_len,
+                                Hq, Hkv, d, page, num_pages, softmax_scale, _ptr(ws),
+                                ws.numel() * ws.element_size(), _stream())
+    _check(rc, ctx)
+    return o
+
+
+def tik_token_logprob(hidden, lm_head, target_ids, inv_temperature: float = 1.0,
+                      ws: Optional[torch.Tensor] = None, logprob: Optional[torch.Tensor] = None,
+                      lse: Optional[torch.Tensor] = None):
+    """hidden [T,H], lm_head [V,H] bf16, target_ids int32 [T] -> logprob fp32 [T]."""
+    ctx = context()
+    bf = torch.bfloat16
+    T, H = hidden.shape
+    V = lm_head.shape[0]
+    need = workspace_bytes(OP_TOKEN_LOGPROB, T, H=H, V=V)
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=hidden.device)
+    if logprob is None:
+        logprob = torch.empty(T, dtype=torch.float32, device=hidden.device)
+    rc = load().tik_token_logprob(ctx, _ptr(hidden, bf), _ptr(lm_head, bf), _ptr(target_ids, torch.int32),
+                                  _ptr(logprob, torch.float32), _ptr(lse, torch.float32), T, H, V,
+                                  inv_temperature, _ptr(ws), ws.numel() * ws.element_size(), _stream())
+    _check(rc, ctx)
+    return logprob

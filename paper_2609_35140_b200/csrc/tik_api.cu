@@ -1,0 +1,367 @@
+// C ABI of libtik: argument checks, tensor maps, grid sizing from host upper bounds, launches.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/tik.h"
+#include "tik_core.cuh"
+#include "tik_internal.h"
+
+namespace tik {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+bool make_tmap_bf16(tik_ctx* ctx, CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+                    const uint64_t* strides_bytes, const uint32_t* box, std::string* err) {
+    cuuint64_t gdim[5], gstr[4];
+    cuuint32_t bdim[5], estr[5];
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        bdim[i] = box[i];
+        estr[i] = 1;
+        if (i > 0) gstr[i - 1] = strides_bytes[i - 1];
+    }
+    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+        out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base), gdim,
+        gstr, bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char buf[256];
+        snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled failed (CUresult %d, rank %d, dims %llu %llu %llu)",
+                 static_cast<int>(r), rank, (unsigned long long)dims[0], (unsigned long long)dims[1],
+                 (unsigned long long)(rank > 2 ? dims[2] : 0));
+        *err = buf;
+        return false;
+    }
+    return true;
+}
+
+static tik_status fail(tik_ctx* ctx, tik_status s, const char* msg) {
+    if (ctx) ctx->last_error = msg;
+    return s;
+}
+static tik_status cuda_fail(tik_ctx* ctx, cudaError_t e, const char* where) {
+    ctx->last_error = std::string(where) + ": " + cudaGetErrorString(e);
+    return TIK_ERR_CUDA;
+}
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool page_ok(int page) { return page == 16 || page == 32 || page == 64 || page == 128; }
+static float scale_to_c(float softmax_scale) { return softmax_scale * LOG2E_F; }
+
+static tik_status check_heads(tik_ctx* ctx, int Hq, int Hkv, int d, float scale) {
+    if (Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return fail(ctx, TIK_ERR_INVALID_ARG, "Hq must be a positive multiple of Hkv");
+    if (!(scale > 0.0f) || !std::isfinite(scale)) return fail(ctx, TIK_ERR_INVALID_ARG, "softmax_scale must be finite and > 0");
+    if (d != 64 && d != 128) return fail(ctx, TIK_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    if (Hq / Hkv > 32) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq/Hkv must be <= 32");
+    return TIK_OK;
+}
+
+}  // namespace tik
+
+using namespace tik;
+
+extern "C" {
+
+tik_status tik_create(tik_ctx** out, int device) {
+    if (!out) return TIK_ERR_INVALID_ARG;
+    *out = nullptr;
+    tik_ctx* ctx = new (std::nothrow) tik_ctx();
+    if (!ctx) return TIK_ERR_CUDA;
+    ctx->device = device;
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    int major = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+    if (e == cudaSuccess && major != 10) {
+        delete ctx;
+        return TIK_ERR_UNSUPPORTED;   // built for sm_100a only
+    }
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, 256);
+    if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, 256);
+    if (e == cudaSuccess) {
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
+        if (e == cudaSuccess && (qres != cudaDriverEntryPointSuccess || !ctx->encode_tiled)) e = cudaErrorNotSupported;
+    }
+    if (e != cudaSuccess) {
+        if (ctx->dev_status) cudaFree(ctx->dev_status);
+        delete ctx;
+        return TIK_ERR_CUDA;
+    }
+    *out = ctx;
+    return TIK_OK;
+}
+
+tik_status tik_destroy(tik_ctx* ctx) {
+    if (!ctx) return TIK_OK;
+    if (ctx->dev_status) cudaFree(ctx->dev_status);
+    delete ctx;
+    return TIK_OK;
+}
+
+const char* tik_status_str(tik_status s) {
+    switch (s) {
+        case TIK_OK: return "ok";
+        case TIK_ERR_INVALID_ARG: return "invalid argument";
+        case TIK_ERR_UNSUPPORTED: return "outside the supported domain";
+        case TIK_ERR_WORKSPACE: return "workspace too small";
+        case TIK_ERR_CUDA: return "CUDA error";
+        default: return "unknown status";
+    }
+}
+
+const char* tik_last_error(const tik_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+const char* tik_contract_id(void) { return TIK_CONTRACT_ID; }
+
+size_t tik_workspace_bytes(int op, int64_t rows_or_batch, int Hq, int Hkv, int d, int64_t max_ctx, int H,
+                           int V) {
+    (void)Hkv;
+    (void)H;
+    if (op == TIK_OP_ATTN_DECODE) {
+        if (rows_or_batch <= 0 || max_ctx <= 0) return 0;
+        const int64_t nchunk = (max_ctx + CHUNK - 1) / CHUNK;
+        return static_cast<size_t>(rows_or_batch) * Hq * nchunk * (d + 2) * sizeof(float);
+    }
+    if (op == TIK_OP_TOKEN_LOGPROB) {
+        if (rows_or_batch <= 0 || V <= 0) return 0;
+        const int64_t nsuper = (V + LP_SUPER - 1) / LP_SUPER;
+        return static_cast<size_t>(rows_or_batch) * (2 * nsuper + 1) * sizeof(float);
+    }
+    return 0;
+}
+
+tik_status tik_device_status(tik_ctx* ctx, void* stream, int* out_flags) {
+    if (!ctx || !out_flags) return TIK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int flags = 0;
+    cudaError_t e = cudaMemcpyAsync(&flags, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->dev_status, 0, sizeof(int), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "tik_device_status");
+    *out_flags = flags;
+    return TIK_OK;
+}
+
+tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const void* v, void* o, float* lse,
+                              const int32_t* cu_seqlens, int S, int64_t total_tokens, int max_seqlen, int Hq,
+                              int Hkv, int d, float softmax_scale, void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (S < 0 || total_tokens < 0 || max_seqlen < 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative size");
+    tik_status s = check_heads(ctx, Hq, Hkv, d, softmax_scale);
+    if (s != TIK_OK) return s;
+    if (S == 0 || total_tokens == 0 || max_seqlen == 0) return TIK_OK;
+    if (!q || !k || !v || !o || !cu_seqlens) return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (total_tokens >= (1ll << 31)) return fail(ctx, TIK_ERR_UNSUPPORTED, "total_tokens must be < 2^31");
+
+    CUtensorMap tmQ, tmK, tmV;
+    std::string err;
+    const uint64_t ud = static_cast<uint64_t>(d);
+    uint64_t qd[3] = {ud, static_cast<uint64_t>(Hq), static_cast<uint64_t>(total_tokens)};
+    uint64_t qs[2] = {ud * 2, ud * 2 * Hq};
+    uint64_t kd[3] = {ud, static_cast<uint64_t>(Hkv), static_cast<uint64_t>(total_tokens)};
+    uint64_t ks[2] = {ud * 2, ud * 2 * Hkv};
+    uint32_t box[3] = {64, 1, 128};
+    if (!make_tmap_bf16(ctx, &tmQ, q, 3, qd, qs, box, &err) || !make_tmap_bf16(ctx, &tmK, k, 3, kd, ks, box, &err) ||
+        !make_tmap_bf16(ctx, &tmV, v, 3, kd, ks, box, &err))
+        return fail(ctx, TIK_ERR_CUDA, err.c_str());
+
+    AttnParams p{};
+    p.o = o;
+    p.lse = lse;
+    p.cu_seqlens = cu_seqlens;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.G = Hq / Hkv;
+    p.c = scale_to_c(softmax_scale);
+    p.dev_status = ctx->dev_status;
+    dim3 grid((max_seqlen + 127) / 128, Hq, S);
+    if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
+    cudaError_t e = launch_attn(d, 0, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_train_fwd");
+}
+
+tik_status tik_kv_cache_write(tik_ctx* ctx, const void* k_new, const void* v_new, const int32_t* cu_seqlens_new,
+                              const int32_t* ctx_lens, void* k_cache, void* v_cache, const int32_t* block_table,
+                              int max_blocks, int S, int64_t total_new, int Hkv, int d, int page_size,
+                              int num_pages, void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (S < 0 || total_new < 0 || max_blocks < 0 || num_pages < 0 || Hkv <= 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative size");
+    if (d != 64 && d != 128) return fail(ctx, TIK_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    if (!page_ok(page_size)) return fail(ctx, TIK_ERR_UNSUPPORTED, "page_size must be 16, 32, 64 or 128");
+    if (S == 0 || total_new == 0) return TIK_OK;
+    if (!k_new || !v_new || !cu_seqlens_new || !ctx_lens || !k_cache || !v_cache || !block_table)
+        return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache))
+        return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (total_new >= (1ll << 31)) return fail(ctx, TIK_ERR_UNSUPPORTED, "total_new must be < 2^31");
+    cudaError_t e = launch_kv_write(k_new, v_new, cu_seqlens_new, ctx_lens, k_cache, v_cache, block_table,
+                                    max_blocks, S, total_new, Hkv, d, page_size, num_pages, ctx->dev_status,
+                                    static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_kv_cache_write");
+}
+
+static tik_status make_cache_maps(tik_ctx* ctx, const void* k_cache, const void* v_cache, int Hkv, int d,
+                                  int page_size, int num_pages, CUtensorMap* tmK, CUtensorMap* tmV) {
+    std::string err;
+    const uint64_t ud = static_cast<uint64_t>(d);
+    uint64_t cd[4] = {ud, static_cast<uint64_t>(page_size), static_cast<uint64_t>(Hkv),
+                      static_cast<uint64_t>(num_pages)};
+    uint64_t cs[3] = {ud * 2, ud * 2 * page_size, ud * 2 * page_size * Hkv};
+    uint32_t box[4] = {64, static_cast<uint32_t>(page_size), 1, 1};
+    if (!make_tmap_bf16(ctx, tmK, k_cache, 4, cd, cs, box, &err) ||
+        !make_tmap_bf16(ctx, tmV, v_cache, 4, cd, cs, box, &err))
+        return fail(ctx, TIK_ERR_CUDA, err.c_str());
+    return TIK_OK;
+}
+
+tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, const int32_t* cu_seqlens_q,
+                            const int32_t* ctx_lens, const void* k_cache, const void* v_cache,
+                            const int32_t* block_table, int max_blocks, int S, int64_t total_q, int max_q_len,
+                            int max_ctx_len, int Hq, int Hkv, int d, int page_size, int num_pages,
+                            float softmax_scale, void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (S < 0 || total_q < 0 || max_q_len < 0 || max_ctx_len < 0 || max_blocks < 0 || num_pages < 0)
+        return fail(ctx, TIK_ERR_INVALID_ARG, "negative size");
+    tik_status s = check_heads(ctx, Hq, Hkv, d, softmax_scale);
+    if (s != TIK_OK) return s;
+    if (!page_ok(page_size)) return fail(ctx, TIK_ERR_UNSUPPORTED, "page_size must be 16, 32, 64 or 128");
+    if (S == 0 || total_q == 0 || max_q_len == 0) return TIK_OK;
+    if (!q || !o || !cu_seqlens_q || !ctx_lens || !k_cache || !v_cache || !block_table || num_pages == 0)
+        return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(q) || !aligned16(o) || !aligned16(k_cache) || !aligned16(v_cache))
+        return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (total_q >= (1ll << 31)) return fail(ctx, TIK_ERR_UNSUPPORTED, "total_q must be < 2^31");
+
+    CUtensorMap tmQ, tmK, tmV;
+    std::string err;
+    const uint64_t ud = static_cast<uint64_t>(d);
+    uint64_t qd[3] = {ud, static_cast<uint64_t>(Hq), static_cast<uint64_t>(total_q)};
+    uint64_t qs[2] = {ud * 2, ud * 2 * Hq};
+    uint32_t box[3] = {64, 1, 128};
+    if (!make_tmap_bf16(ctx, &tmQ, q, 3, qd, qs, box, &err)) return fail(ctx, TIK_ERR_CUDA, err.c_str());
+    s = make_cache_maps(ctx, k_cache, v_cache, Hkv, d, page_size, num_pages, &tmK, &tmV);
+    if (s != TIK_OK) return s;
+
+    AttnParams p{};
+    p.o = o;
+    p.lse = lse;
+    p.cu_seqlens = cu_seqlens_q;
+    p.ctx_lens = ctx_lens;
+    p.block_table = block_table;
+    p.max_blocks = max_blocks;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.G = Hq / Hkv;
+    p.page_size = page_size;
+    p.pages_per_tile = 128 / page_size;
+    p.num_pages = num_pages;
+    p.c = scale_to_c(softmax_scale);
+    p.dev_status = ctx->dev_status;
+    // query tiles are aligned to absolute positions: an unaligned start adds one tile
+    dim3 grid((max_q_len + 127) / 128 + 1, Hq, S);
+    if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
+    cudaError_t e = launch_attn(d, 1, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_prefill");
+}
+
+tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, const int32_t* ctx_lens,
+                           const void* k_cache, const void* v_cache, const int32_t* block_table, int max_blocks,
+                           int B, int max_ctx_len, int Hq, int Hkv, int d, int page_size, int num_pages,
+                           float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (B < 0 || max_ctx_len < 0 || max_blocks < 0 || num_pages < 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative size");
+    tik_status s = check_heads(ctx, Hq, Hkv, d, softmax_scale);
+    if (s != TIK_OK) return s;
+    if (!page_ok(page_size)) return fail(ctx, TIK_ERR_UNSUPPORTED, "page_size must be 16, 32, 64 or 128");
+    if (B == 0 || max_ctx_len == 0) return TIK_OK;
+    if (!q || !o || !ctx_lens || !k_cache || !v_cache || !block_table || num_pages == 0)
+        return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(q) || !aligned16(o) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
+        return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    const size_t need = tik_workspace_bytes(TIK_OP_ATTN_DECODE, B, Hq, Hkv, d, max_ctx_len, 0, 0);
+    if (!ws || ws_bytes < need) return fail(ctx, TIK_ERR_WORKSPACE, "decode workspace too small");
+
+    CUtensorMap tmQ, tmK, tmV;
+    std::string err;
+    const uint64_t ud = static_cast<uint64_t>(d);
+    const int G = Hq / Hkv;
+    uint64_t qd[3] = {ud, static_cast<uint64_t>(Hq), static_cast<uint64_t>(B)};
+    uint64_t qs[2] = {ud * 2, ud * 2 * Hq};
+    uint32_t box[3] = {64, static_cast<uint32_t>(G), 1};
+    if (!make_tmap_bf16(ctx, &tmQ, q, 3, qd, qs, box, &err)) return fail(ctx, TIK_ERR_CUDA, err.c_str());
+    s = make_cache_maps(ctx, k_cache, v_cache, Hkv, d, page_size, num_pages, &tmK, &tmV);
+    if (s != TIK_OK) return s;
+
+    const int nchunk = (max_ctx_len + CHUNK - 1) / CHUNK;
+    AttnParams p{};
+    p.o = o;
+    p.lse = lse;
+    p.ctx_lens = ctx_lens;
+    p.block_table = block_table;
+    p.max_blocks = max_blocks;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.G = G;
+    p.page_size = page_size;
+    p.pages_per_tile = 128 / page_size;
+    p.num_pages = num_pages;
+    p.c = scale_to_c(softmax_scale);
+    p.nchunk_max = nchunk;
+    p.part_o = static_cast<float*>(ws);
+    p.part_ml = p.part_o + static_cast<size_t>(B) * Hq * nchunk * d;
+    p.dev_status = ctx->dev_status;
+    dim3 grid(nchunk, Hkv, B);
+    if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hkv and B must be <= 65535");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_attn(d, 2, grid, tmQ, tmK, tmV, p, st);
+    if (e == cudaSuccess) e = launch_combine(d, p, B, st);
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_decode");
+}
+
+tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_head, const int32_t* target_ids,
+                             float* logprob, float* lse, int64_t T, int H, int V, float inv_temperature, void* ws,
+                             size_t ws_bytes, void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (T < 0 || H <= 0 || V <= 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative or zero size");
+    if (!(inv_temperature > 0.0f) || !std::isfinite(inv_temperature))
+        return fail(ctx, TIK_ERR_INVALID_ARG, "inv_temperature must be finite and > 0");
+    if (H % 64 != 0) return fail(ctx, TIK_ERR_UNSUPPORTED, "H must be a multiple of 64");
+    if (T == 0) return TIK_OK;
+    if (!hidden || !lm_head || !target_ids || !logprob) return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(hidden) || !aligned16(lm_head) || !aligned16(ws)) return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (T >= (1ll << 31) - 128) return fail(ctx, TIK_ERR_UNSUPPORTED, "T must be < 2^31 - 128");
+    const size_t need = tik_workspace_bytes(TIK_OP_TOKEN_LOGPROB, T, 0, 0, 0, 0, H, V);
+    if (!ws || ws_bytes < need) return fail(ctx, TIK_ERR_WORKSPACE, "log-prob workspace too small");
+
+    CUtensorMap tmA, tmB;
+    std::string err;
+    uint64_t ad[2] = {static_cast<uint64_t>(H), static_cast<uint64_t>(T)};
+    uint64_t bd[2] = {static_cast<uint64_t>(H), static_cast<uint64_t>(V)};
+    uint64_t st1[1] = {static_cast<uint64_t>(H) * 2};
+    uint32_t box[2] = {64, 128};
+    if (!make_tmap_bf16(ctx, &tmA, hidden, 2, ad, st1, box, &err) ||
+        !make_tmap_bf16(ctx, &tmB, lm_head, 2, bd, st1, box, &err))
+        return fail(ctx, TIK_ERR_CUDA, err.c_str());
+
+    LogprobParams p{};
+    p.target = target_ids;
+    p.logprob = logprob;
+    p.lse = lse;
+    p.T = T;
+    p.H = H;
+    p.V = V;
+    p.nsuper = (V + LP_SUPER - 1) / LP_SUPER;
+    p.part_ml = static_cast<float*>(ws);
+    p.z_target = p.part_ml + static_cast<size_t>(T) * p.nsuper * 2;
+    p.inv_temperature = inv_temperature;
+    p.dev_status = ctx->dev_status;
+    cudaError_t e = launch_logprob(tmA, tmB, p, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_token_logprob");
+}
+
+}  // extern "C"

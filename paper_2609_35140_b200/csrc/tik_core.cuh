@@ -1,0 +1,118 @@
+// The numerical contract shared by every regime (packed train-forward, paged prefill,
+// paged decode, split-KV combine) and by the log-probability kernels.
+//
+// Section 5.2 of the paper lists what decides the bits of unified attention: the
+// reduction orders of QK^T, PV, online softmax and final normalisation; where and in
+// which precision scaling and masking happen; the exact exp / reciprocal instructions
+// and flush-to-zero behaviour; the bf16<->fp32 conversion points and the order of
+// rescale, update and normalise.  Section 3.2 adds that KV-tile boundaries determine
+// rescaling, P rounding and PV order.  This header fixes each of those once; all
+// kernels call these functions and nothing else for that arithmetic.
+//
+//   * KV tile: 128 keys at absolute positions [128 j, 128 j + 128), ascending j.
+//   * Chunk: 2048 keys (16 tiles), absolute-aligned.  The running state (m, l, O) is
+//     reset at every chunk start in every regime; chunks are folded in ascending order.
+//   * Scores: fp32 accumulators of a K=16 tcgen05 MMA chain (ascending over head_dim).
+//   * c = softmax_scale * log2(e), one fp32 multiply on the host.
+//   * Mask: select -inf where key position > query position (no arithmetic on masked
+//     scores, so masked K contents never matter).
+//   * Per tile and row: m' = max(m, tile max); p = ex2.approx.ftz(fma(s, c, -(m' * c)));
+//     row sum in the fixed 8-chain shape below; alpha = ex2.approx.ftz((m - m') * c);
+//     l = fma(l, alpha, rowsum); O = O * alpha with a non-flushing IEEE multiply (so
+//     skipping it when alpha == 1.0f is bit-neutral); P rounded to bf16 (RNE) for the PV
+//     MMA while l sums the unrounded fp32 p.
+//   * Finalise: o = O * rcp.rn(l), rounded to bf16 (RNE).
+#pragma once
+#include <cuda_bf16.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+namespace tik {
+
+constexpr int BN = 128;               // keys per KV tile
+constexpr int BM = 128;               // query rows per MMA tile
+constexpr int CHUNK = 2048;           // keys per split chunk
+constexpr int TILES_PER_CHUNK = CHUNK / BN;
+constexpr float LOG2E_F = 1.44269504088896340736f;
+constexpr float LN2_F = 0.69314718055994530942f;
+constexpr int LP_TILE = 128;          // vocabulary columns per log-sum-exp tile
+constexpr int LP_SUPER = 1024;        // vocabulary columns per super-chunk (8 tiles)
+
+#define TIK_CONTRACT_ID "tik1-BN128-CH2048-M128N128K16-ex2ftz-sum8-LP128x1024"
+
+__device__ __forceinline__ float ex2_ftz(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Running row sum in a fixed shape: chain index = 4 * (col / 64) + ((col / 2) % 4); every
+// chain adds its columns in ascending order; the eight chains are combined as
+// ((a0+a1)+(a2+a3)) + ((a4+a5)+(a6+a7)).  The shape lets a row be summed by one thread,
+// by two threads owning 64 columns each, or by four threads owning interleaved column
+// pairs, with identical bits.
+struct RowSum8 {
+    float a[8];
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] = 0.0f;
+    }
+    __device__ __forceinline__ float total() const {
+        const float lo = __fadd_rn(__fadd_rn(a[0], a[1]), __fadd_rn(a[2], a[3]));
+        const float hi = __fadd_rn(__fadd_rn(a[4], a[5]), __fadd_rn(a[6], a[7]));
+        return __fadd_rn(lo, hi);
+    }
+};
+// `col` must be a compile-time constant after unrolling.
+__device__ __forceinline__ void rowsum_add(RowSum8& s, int col, float p) {
+    const int chain = ((col >> 6) << 2) | ((col >> 1) & 3);
+    s.a[chain] = __fadd_rn(s.a[chain], p);
+}
+
+// exponent argument of one score: s * c - mc, one fused multiply-add.
+__device__ __forceinline__ float softmax_p(float s, float c, float neg_mc) {
+    return ex2_ftz(__fmaf_rn(s, c, neg_mc));
+}
+// rescale factor when the row maximum moves from m_old to m_new (m_new >= m_old).
+// Subtract first: m_new == m_old gives ex2(0) = 1.0f exactly; m_old = -inf gives 0.
+__device__ __forceinline__ float softmax_alpha(float m_old, float m_new, float c) {
+    return ex2_ftz(__fmul_rn(__fsub_rn(m_old, m_new), c));
+}
+__device__ __forceinline__ float rescale_o(float o, float alpha) { return __fmul_rn(o, alpha); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits), RNE
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+
+// Fold chunk state (m_c, l_c, O_c) into the global state (M, L, O).  The global state is
+// initialised by copying chunk 0; chunks 1, 2, ... are folded in ascending order.
+struct FoldCoef {
+    float A, B, M_new;
+};
+__device__ __forceinline__ FoldCoef fold_coef(float M, float m_c, float c) {
+    FoldCoef f;
+    f.M_new = fmaxf(M, m_c);
+    f.A = ex2_ftz(__fmul_rn(__fsub_rn(M, f.M_new), c));
+    f.B = ex2_ftz(__fmul_rn(__fsub_rn(m_c, f.M_new), c));
+    return f;
+}
+__device__ __forceinline__ float fold_value(float X, float x_c, const FoldCoef& f) {
+    return __fmaf_rn(X, f.A, __fmul_rn(x_c, f.B));
+}
+
+__device__ __forceinline__ float finalize_inv(float L) { return __frcp_rn(L); }
+__device__ __forceinline__ float finalize_o(float O, float inv) { return __fmul_rn(O, inv); }
+// natural-log log-sum-exp of the scaled scores: (M * c + log2 L) * ln 2
+__device__ __forceinline__ float finalize_lse(float M, float L, float c) {
+    return __fmul_rn(__fadd_rn(__fmul_rn(M, c), log2f(L)), LN2_F);
+}
+
+// ---- log-probability: tile (m, l) with natural-exponent semantics via exp2 ----------
+// l_j = sum ex2(fma(z, log2e, -(m_j * log2e))) in the RowSum8 shape; tiles and super-chunks
+// are folded sequentially in ascending column order with fold_coef(c = log2e).
+__device__ __forceinline__ float lp_lse(float M, float L) {
+    return __fadd_rn(M, __fmul_rn(log2f(L), LN2_F));
+}
+
+}  // namespace tik

@@ -1,0 +1,65 @@
+// Host-side declarations shared by the translation units of libtik (not part of the ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+
+struct tik_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int* dev_status = nullptr;          // one int of device flags (TIK_DEV_*)
+    void* encode_tiled = nullptr;       // cuTensorMapEncodeTiled from the driver
+    std::string last_error;
+};
+
+namespace tik {
+
+// Builds a bf16 tiled tensor map with 128-byte swizzle; dims/box innermost first, strides
+// in bytes for dims 1..rank-1.  Returns false (and fills err) on failure.
+bool make_tmap_bf16(tik_ctx* ctx, CUtensorMap* out, const void* base, int rank,
+                    const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box,
+                    std::string* err);
+
+struct AttnParams {
+    void* o;                     // bf16 output rows
+    float* lse;                  // optional
+    const int32_t* cu_seqlens;   // train: per sequence; prefill: per sequence, query tokens
+    const int32_t* ctx_lens;     // prefill / decode
+    const int32_t* block_table;  // prefill / decode
+    int max_blocks;
+    int Hq, Hkv, G;
+    int page_size, pages_per_tile, num_pages;
+    float c;                     // softmax_scale * log2(e)
+    float* part_o;               // decode: [B][Hq][nchunk_max][d]
+    float* part_ml;              // decode: [B][Hq][nchunk_max][2]
+    int nchunk_max;
+    int* dev_status;
+};
+
+// mode: 0 train (packed K/V), 1 prefill (paged K/V), 2 decode (paged K/V, chunk partials)
+cudaError_t launch_attn(int d, int mode, dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                        const CUtensorMap& tmV, const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_combine(int d, const AttnParams& p, int B, cudaStream_t stream);
+cudaError_t launch_kv_write(const void* k_new, const void* v_new, const int32_t* cu_new,
+                            const int32_t* ctx_lens, void* k_cache, void* v_cache,
+                            const int32_t* block_table, int max_blocks, int S, int64_t total_new,
+                            int Hkv, int d, int page_size, int num_pages, int* dev_status,
+                            cudaStream_t stream);
+
+struct LogprobParams {
+    const int32_t* target;
+    float* logprob;
+    float* lse;                  // optional
+    float* part_ml;              // [T][nsuper][2]
+    float* z_target;             // [T]
+    int64_t T;
+    int H, V, nsuper;
+    float inv_temperature;
+    int* dev_status;
+};
+cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p,
+                           cudaStream_t stream);
+
+}  // namespace tik

@@ -1,0 +1,249 @@
+// Token log-probability for sm_100a: lm_head GEMM on tcgen05 fused with a chunked
+// log-sum-exp over the vocabulary and the target-logit gather.  The fp32 logits live only
+// in TMEM; nothing of size T x V is ever written.
+//
+// One CTA = (128-token tile, 1024-column super-chunk).  For each of the (up to) eight
+// 128-column tiles of the super-chunk, a TMA warp streams 64-wide K slices of hidden and
+// lm_head through a shared-memory ring, an MMA warp accumulates the whole K range in
+// ascending order into one of two TMEM accumulators (no split-K), and four epilogue warps
+// (one thread per token row) reduce the finished tile to (max, sum of exp) with the fixed
+// row-sum shape, fold it into the super-chunk's running pair, and pick the target logit if
+// this tile owns its column.  A finish kernel folds the super-chunk pairs of every token in
+// ascending order and writes logprob = z_target - logsumexp.
+#include "tik_core.cuh"
+#include "tik_internal.h"
+#include "tik_ptx.cuh"
+
+namespace tik {
+
+namespace lp {
+constexpr int STAGES = 6;
+constexpr uint32_t A_BYTES = 128 * 128;      // 128 token rows x 64 bf16
+constexpr uint32_t B_BYTES = 128 * 128;      // 128 vocab rows x 64 bf16
+constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t OFF_BAR = STAGES * STAGE_BYTES;
+constexpr uint32_t BYTES = OFF_BAR + 256;
+constexpr uint32_t ALLOC = BYTES + 1024;
+constexpr int BAND = 32;                     // token tiles per L2 band
+constexpr int THREADS = 192;                 // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+}  // namespace lp
+
+__global__ void __launch_bounds__(lp::THREADS, 1)
+logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const LogprobParams p) {
+    using namespace lp;
+    constexpr uint32_t TMEM_COLS = 256;      // two 128-column accumulators
+    constexpr uint32_t IDESC = mma_idesc_bf16(128, 128, false);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // raster: bands of BAND token tiles; within a band the token tile varies fastest so the
+    // CTAs in flight share one lm_head super-chunk and the band's hidden rows stay in L2
+    const int ntile = static_cast<int>((p.T + 127) / 128);
+    const long long per_band = static_cast<long long>(BAND) * p.nsuper;
+    const int band = static_cast<int>(blockIdx.x / per_band);
+    const int band_tiles = min(BAND, ntile - band * BAND);
+    const long long rem = blockIdx.x - band * per_band;
+    // (blockIdx.x enumerates BAND * nsuper slots per band; slots beyond a short last band exit)
+    const int sup = static_cast<int>(rem / BAND);
+    const int tile_in_band = static_cast<int>(rem % BAND);
+    if (tile_in_band >= band_tiles) return;
+    const int tok0 = (band * BAND + tile_in_band) * 128;
+    const int col_base = sup * LP_SUPER;
+    const int n_nt = min(LP_SUPER / LP_TILE, (p.V - col_base + LP_TILE - 1) / LP_TILE);
+    const int n_kb = p.H / 64;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t* smem = smem_raw + pad;
+    const uint32_t sbase = raw_addr + pad;
+    const uint32_t bar_full = sbase + OFF_BAR;               // STAGES barriers
+    const uint32_t bar_empty = bar_full + 8 * STAGES;        // STAGES barriers
+    const uint32_t bar_acc_full = bar_empty + 8 * STAGES;    // 2
+    const uint32_t bar_acc_empty = bar_acc_full + 16;        // 2
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 8 * (2 * STAGES + 4));
+    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + OFF_BAR + 8 * (2 * STAGES + 4) + 4);
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, 128);
+        }
+        *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int nt = 0; nt < n_nt; ++nt) {
+                const int col0 = col_base + nt * LP_TILE;
+                for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t use = it / STAGES;
+                    if (use > 0) mbar_wait(bar_empty + 8 * s, (use - 1) & 1, abort_word, p.dev_status);
+                    mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
+                    tma_load_2d(sbase + s * STAGE_BYTES, &tmA, bar_full + 8 * s, kb * 64, tok0);
+                    tma_load_2d(sbase + s * STAGE_BYTES + A_BYTES, &tmB, bar_full + 8 * s, kb * 64, col0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int nt = 0; nt < n_nt; ++nt) {
+                const int buf = nt & 1;
+                const uint32_t use = nt >> 1;
+                if (use > 0) mbar_wait(bar_acc_empty + 8 * buf, (use - 1) & 1, abort_word, p.dev_status);
+                tc_fence_after();
+                for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    mbar_wait(bar_full + 8 * s, (it / STAGES) & 1, abort_word, p.dev_status);
+                    tc_fence_after();
+                    const uint32_t a0 = sbase + s * STAGE_BYTES, b0 = a0 + A_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ss(tmem + buf * 128, smem_desc_sw128(a0 + ks * 32, 0, 1024),
+                               smem_desc_sw128(b0 + ks * 32, 0, 1024), IDESC, (kb | ks) ? 1u : 0u);
+                    mma_commit(bar_empty + 8 * s);
+                }
+                mma_commit(bar_acc_full + 8 * buf);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;                      // TMEM lane quarter of this warp
+        const int row = quarter * 32 + lane;
+        const long long t = static_cast<long long>(tok0) + row;
+        const bool row_valid = t < p.T;
+        const int target = row_valid ? p.target[t] : -1;
+        const float it_scale = p.inv_temperature;
+        float M = -CUDART_INF_F, Lsum = 0.0f;
+        for (int nt = 0; nt < n_nt; ++nt) {
+            const int buf = nt & 1;
+            const int col0 = col_base + nt * LP_TILE;
+            mbar_wait(bar_acc_full + 8 * buf, (nt >> 1) & 1, abort_word, p.dev_status);
+            tc_fence_after();
+            const uint32_t taddr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 128;
+            const int vmax = p.V - 1 - col0;               // columns > vmax are past the vocabulary
+            float mt = -CUDART_INF_F;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t v[32];
+                tmem_ld32(taddr + 32 * cc, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    float z = __fmul_rn(__uint_as_float(v[i]), it_scale);
+                    if (32 * cc + i > vmax) z = -CUDART_INF_F;
+                    mt = fmaxf(mt, z);
+                }
+            }
+            const float neg_mc = -__fmul_rn(mt, LOG2E_F);
+            const int tcol = target - col0;                // in [0,128) when this tile owns the target
+            float zt = 0.0f;
+            RowSum8 rs;
+            rs.reset();
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t v[32];
+                tmem_ld32(taddr + 32 * cc, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float z = __fmul_rn(__uint_as_float(v[i]), it_scale);
+                    float e = softmax_p(z, LOG2E_F, neg_mc);
+                    if (32 * cc + i > vmax) e = 0.0f;
+                    rowsum_add(rs, 32 * cc + i, e);
+                    if (32 * cc + i == tcol) zt = z;
+                }
+            }
+            // all TMEM reads of this accumulator are done: hand it back to the MMA warp
+            tc_fence_before();
+            mbar_arrive(bar_acc_empty + 8 * buf);
+            const float lt = rs.total();
+            if (nt == 0) {
+                M = mt;
+                Lsum = lt;
+            } else {
+                const FoldCoef f = fold_coef(M, mt, LOG2E_F);
+                Lsum = fold_value(Lsum, lt, f);
+                M = f.M_new;
+            }
+            if (row_valid && tcol >= 0 && tcol < LP_TILE && target < p.V) p.z_target[t] = zt;
+        }
+        if (row_valid) {
+            p.part_ml[2 * (t * p.nsuper + sup)] = M;
+            p.part_ml[2 * (t * p.nsuper + sup) + 1] = Lsum;
+        }
+    }
+
+    if (*abort_word) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) {
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// One thread per token: fold the super-chunk pairs in ascending order, write the result.
+__global__ void __launch_bounds__(256) logprob_finish_kernel(const LogprobParams p) {
+    const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t >= p.T) return;
+    const float* ml = p.part_ml + 2 * t * p.nsuper;
+    float M = ml[0], Lsum = ml[1];
+    for (int s = 1; s < p.nsuper; ++s) {
+        const FoldCoef f = fold_coef(M, ml[2 * s], LOG2E_F);
+        Lsum = fold_value(Lsum, ml[2 * s + 1], f);
+        M = f.M_new;
+    }
+    const float lse = lp_lse(M, Lsum);
+    if (p.lse) p.lse[t] = lse;
+    const int target = p.target[t];
+    if (target < 0 || target >= p.V) {
+        atomicOr(p.dev_status, TIK_DEV_BAD_TARGET);
+        p.logprob[t] = CUDART_NAN_F;
+    } else {
+        p.logprob[t] = __fsub_rn(p.z_target[t], lse);
+    }
+}
+
+cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p,
+                           cudaStream_t stream) {
+    if (p.T <= 0) return cudaSuccess;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(logprob_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(lp::ALLOC));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const long long ntile = (p.T + 127) / 128;
+    const long long nband = (ntile + lp::BAND - 1) / lp::BAND;
+    const long long grid = nband * lp::BAND * p.nsuper;
+    logprob_kernel<<<static_cast<unsigned>(grid), lp::THREADS, lp::ALLOC, stream>>>(tmA, tmB, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    logprob_finish_kernel<<<static_cast<unsigned>((p.T + 255) / 256), 256, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace tik

@@ -1,0 +1,123 @@
+"""GPU parity: the three attention regimes against the CPU oracle (tolerance) and against
+each other (zero differing bits), through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_35140_b200 import synth
+from gpu_common import ATTN_TOL, Rollout, bits, count_diff
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tik():
+    from paper_2609_35140_b200 import binding
+    binding.load()
+    yield binding
+    assert binding.device_status() == 0
+
+
+def _oracle_packed(w, q, k, v):
+    out, _ = oracle.attn_packed(q.float().cpu().numpy(), k.float().cpu().numpy(),
+                                v.float().cpu().numpy(), w.cu_seqlens(), w.softmax_scale)
+    return out
+
+
+def _train(tik, w, q, k, v, cu, max_seqlen=None, lse=None):
+    return tik.tik_attn_train_fwd(q, k, v, cu, max_seqlen or max(w.seq_lens), w.softmax_scale, lse=lse)
+
+
+WORKLOADS = {
+    "tiny": lambda: synth.get_workload(0),
+    "d128_ragged": lambda: synth.custom_workload([100, 129, 1, 300], [57, 200, 3, 213], 8, 2, 128, 64),
+    "d64_page32": lambda: synth.custom_workload([33, 250], [95, 140], 6, 3, 64, 32),
+    "d128_page16_g1": lambda: synth.custom_workload([70], [186], 2, 2, 128, 16),
+    "d128_page128_g16": lambda: synth.custom_workload([128, 5], [130, 250], 16, 1, 128, 128),
+}
+
+
+@pytest.mark.parametrize("name", list(WORKLOADS))
+def test_train_fwd_matches_oracle(tik, name):
+    w = WORKLOADS[name]()
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    lse = torch.full((w.total_tokens, w.Hq), -1.0, dtype=torch.float32, device="cuda")
+    o = _train(tik, w, q, k, v, cu, lse=lse)
+    ref, ref_lse = oracle.attn_packed(q.float().cpu().numpy(), k.float().cpu().numpy(),
+                                      v.float().cpu().numpy(), w.cu_seqlens(), w.softmax_scale)
+    err = np.abs(o.float().cpu().numpy() - ref).max()
+    assert err <= ATTN_TOL, err
+    assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 1e-3
+    # position 0 of every sequence attends one key: the output is that V row, bit for bit
+    cu_h = w.cu_seqlens()
+    for s in range(w.S):
+        for h in range(w.Hq):
+            assert torch.equal(bits(o[cu_h[s], h]), bits(v[cu_h[s], h // w.G]))
+
+
+@pytest.mark.parametrize("name", list(WORKLOADS))
+def test_rollout_replay_is_bit_identical_to_train_fwd(tik, name):
+    """Eq. 1: update-forward rows == prefill rows || decode rows, at every position."""
+    w = WORKLOADS[name]()
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    o_train = _train(tik, w, q, k, v, cu)
+    layout = synth.make_paged_layout(w)
+    o_roll = Rollout(tik, w, q, k, v, layout).replay()
+    assert count_diff(o_train, o_roll) == 0
+    ref = _oracle_packed(w, q, k, v)
+    assert np.abs(o_roll.float().cpu().numpy() - ref).max() <= ATTN_TOL
+
+
+def test_multi_chunk_sequences(tik):
+    """Contexts longer than one 2048-key chunk: in-kernel fold (train/prefill) and the
+    split-KV combine (decode) agree bit for bit and with the oracle."""
+    w = synth.custom_workload([2100, 1500], [2200, 700], 4, 2, 128, 64)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    o_train = _train(tik, w, q, k, v, cu)
+    ref = _oracle_packed(w, q, k, v)
+    assert np.abs(o_train.float().cpu().numpy() - ref).max() <= ATTN_TOL
+    layout = synth.make_paged_layout(w)
+    ro = Rollout(tik, w, q, k, v, layout)
+    rows, o = ro.prefill()
+    assert count_diff(o, o_train[rows]) == 0
+    # fill the rest of the cache, then decode a few late positions directly
+    cu_h = w.cu_seqlens()
+    rest = [(s, w.prompt_lens[s], w.seq_lens[s]) for s in range(w.S)]
+    rows2, o2 = ro.prefill(seqs=[r[0] for r in rest], start=[r[1] for r in rest], stop=[r[2] for r in rest])
+    assert count_diff(o2, o_train[rows2]) == 0
+    for pos in ([2047, 1499], [2048, 2047], [4299, 2199], [4096, 2048]):
+        # K/V of those positions are already in the cache; rewriting them is idempotent
+        rows3, o3 = ro.decode_step([0, 1], pos)
+        assert count_diff(o3, o_train[rows3]) == 0, pos
+
+
+def test_kv_cache_write_is_exact(tik):
+    w = synth.get_workload(0)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    layout = synth.make_paged_layout(w)
+    ro = Rollout(tik, w, q, k, v, layout, dirty=3.0)
+    upto = [40, 64]
+    ro.prefill(stop=upto)
+    kc_ref, vc_ref = synth.fill_paged_cache(w, layout, k, v, upto=upto, fill=3.0)
+    assert torch.equal(bits(ro.kc), bits(kc_ref)) and torch.equal(bits(ro.vc), bits(vc_ref))
+
+
+def test_invalid_arguments_are_rejected(tik):
+    w = synth.get_workload(0)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    with pytest.raises(tik.TikError):
+        tik.tik_attn_train_fwd(q[:, :3].contiguous(), k, v, cu, 160, w.softmax_scale)      # Hq % Hkv
+    with pytest.raises(tik.TikError):
+        tik.tik_attn_train_fwd(q, k, v, cu, 160, -1.0)
+    q96 = torch.zeros(4, 4, 96, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(tik.TikError):
+        tik.tik_attn_train_fwd(q96, q96[:, :1].contiguous(), q96[:, :1].contiguous(),
+                               torch.tensor([0, 4], dtype=torch.int32, device="cuda"), 4, 0.1)
+    layout = synth.make_paged_layout(w)
+    kc, vc = synth.fill_paged_cache(w, layout, k, v)
+    bt = torch.from_numpy(layout.block_table).cuda()
+    ctx = torch.tensor(w.seq_lens, dtype=torch.int32, device="cuda")
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(tik.TikError):
+        tik.tik_attn_decode(q[:2].contiguous(), ctx, kc, vc, bt, 160, w.softmax_scale, ws=small)
