@@ -147,13 +147,13 @@ def _randn_bf16(shape, gen, device, std=1.0, chunk_rows=1 << 16):
     return out
 
 
-def make_qkv(w: Workload, device="cpu") -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor,
-                                                   torch.Tensor]:
+def make_qkv(w: Workload, device="cpu", seed_offset: int = 0) -> Tuple[
+        torch.Tensor, torch.Tensor, torch.Tensor, torch.Tensor]:
     """Packed q [tot,Hq,d], k, v [tot,Hkv,d] (bf16) and cu_seqlens (int32).
 
     Sequences of one group carry identical prompt rows (a shared prompt)."""
     gen = torch.Generator(device=device)
-    gen.manual_seed(w.seed)
+    gen.manual_seed(w.seed + seed_offset)
     tot = w.total_tokens
     q = _randn_bf16((tot, w.Hq, w.d), gen, device)
     k = _randn_bf16((tot, w.Hkv, w.d), gen, device)
@@ -240,10 +240,10 @@ def fill_paged_cache(w: Workload, layout: PagedLayout, k: torch.Tensor, v: torch
     return kc, vc
 
 
-def make_logprob_inputs(w: Workload, device="cpu", T: Optional[int] = None):
+def make_logprob_inputs(w: Workload, device="cpu", T: Optional[int] = None, seed_offset: int = 0):
     """hidden [T,H] ~ N(0,1), lm_head [V,H] ~ N(0, 0.02) (bf16), target ids uniform (int32)."""
     gen = torch.Generator(device=device)
-    gen.manual_seed(w.seed + 104729)
+    gen.manual_seed(w.seed + 104729 + seed_offset)
     T = w.response_tokens if T is None else T
     hidden = _randn_bf16((T, w.hidden), gen, device)
     W = _randn_bf16((w.vocab, w.hidden), gen, device, std=0.02, chunk_rows=1 << 14)

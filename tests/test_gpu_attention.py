@@ -106,8 +106,9 @@ def test_kv_cache_write_is_exact(tik):
 def test_invalid_arguments_are_rejected(tik):
     w = synth.get_workload(0)
     q, k, v, cu = synth.make_qkv(w, "cuda")
+    k2 = torch.cat([k, k], 1).contiguous()
     with pytest.raises(tik.TikError):
-        tik.tik_attn_train_fwd(q[:, :3].contiguous(), k, v, cu, 160, w.softmax_scale)      # Hq % Hkv
+        tik.tik_attn_train_fwd(q[:, :3].contiguous(), k2, k2, cu, 160, w.softmax_scale)    # Hq % Hkv
     with pytest.raises(tik.TikError):
         tik.tik_attn_train_fwd(q, k, v, cu, 160, -1.0)
     q96 = torch.zeros(4, 4, 96, dtype=torch.bfloat16, device="cuda")
