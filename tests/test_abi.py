@@ -1,0 +1,41 @@
+"""The C-ABI library loads without a GPU and exports every function the header declares."""
+import ctypes
+import os
+import re
+
+from paper_2609_35140_b200 import build as tik_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "tik.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(tik_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_declares_the_entry_points():
+    names = _declared_functions()
+    for required in ("tik_attn_train_fwd", "tik_attn_prefill", "tik_attn_decode", "tik_token_logprob",
+                     "tik_kv_cache_write", "tik_create", "tik_destroy", "tik_workspace_bytes"):
+        assert required in names
+
+
+def test_library_exports_every_declared_symbol():
+    path = tik_build.build()
+    lib = ctypes.CDLL(path)
+    for name in _declared_functions():
+        assert hasattr(lib, name), name
+
+
+def test_host_only_calls_work_without_a_gpu():
+    from paper_2609_35140_b200 import binding
+    assert binding.contract_id().startswith("tik1-")
+    lib = binding.load()
+    assert lib.tik_status_str(0) == b"ok"
+    assert lib.tik_status_str(-3) == b"workspace too small"
+    # decode scratch: B * Hq * chunks * (d + 2) floats; log-prob: T * (2 * super-chunks + 1) floats
+    assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 16384) == 16 * 32 * 8 * 130 * 4
+    assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 2049) == 16 * 32 * 2 * 130 * 4
+    assert binding.workspace_bytes(binding.OP_TOKEN_LOGPROB, 1000, H=4096, V=151936) == 1000 * (2 * 149 + 1) * 4
+    assert binding.workspace_bytes(binding.OP_ATTN_TRAIN_FWD, 1000, 8, 2, 128, 4096) == 0
