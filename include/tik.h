@@ -133,6 +133,31 @@ tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_he
                              int H, int V, float inv_temperature, void* ws, size_t ws_bytes,
                              void* stream);
 
+/* Decode attention without any allocation (the paper has no counterpart; this variant
+ * exists for deployments of this library).  Same arguments, kernels and output bits as
+ * tik_attn_decode, but it takes no tik_ctx and no workspace: the split-KV scratch is a
+ * fixed __device__ array of TIK_STATIC_SCRATCH_BYTES inside the library, resident on every
+ * GPU that loads the library until the process exits.  Meant for callers that cannot call
+ * cudaMalloc: a server whose KV-cache pool already owns all free device memory, or a decode
+ * loop that must avoid the device-wide synchronisation of cudaMalloc/cudaFree.
+ *   - Needs B * Hq * ceil(max_ctx_len/2048) * (d+2) * 4 <= TIK_STATIC_SCRATCH_BYTES,
+ *     otherwise returns TIK_ERR_WORKSPACE and launches nothing.
+ *   - Works on the current CUDA device.  The first call on each device resolves the
+ *     scratch's device address and the driver's tensor-map encoder (host-side set-up, no
+ *     allocation); make that first call before any stream capture.
+ *   - All calls on a device share the one scratch array: two calls whose kernels may overlap
+ *     on the GPU (different streams) race on it.  Issue them on one stream or order them.
+ *   - dev_flags: optional device int that receives TIK_DEV_* flags (OR-ed in; the caller
+ *     zeroes and reads it).  NULL sends the flags to a word inside the library.
+ *   - No error text is kept (there is no context): only the status code is returned. */
+#define TIK_STATIC_SCRATCH_BYTES (8u << 20)
+tik_status tik_attn_decode_static(const void* q, void* o, float* lse, const int32_t* ctx_lens,
+                                  const void* k_cache, const void* v_cache,
+                                  const int32_t* block_table, int max_blocks, int B,
+                                  int max_ctx_len, int Hq, int Hkv, int d, int page_size,
+                                  int num_pages, float softmax_scale, int* dev_flags,
+                                  void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -58,6 +58,9 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.tik_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32,
                                     f32, vp, sz, vp]
     lib.tik_token_logprob.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, f32, vp, sz, vp]
+    lib.tik_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
+                                           i32, f32, vp, vp]
+    lib.tik_attn_decode_static.restype = i32
     for name in ("tik_create", "tik_destroy", "tik_device_status", "tik_attn_train_fwd",
                  "tik_kv_cache_write", "tik_attn_prefill", "tik_attn_decode", "tik_token_logprob"):
         getattr(lib, name).restype = i32
@@ -206,3 +209,24 @@ def tik_token_logprob(hidden, lm_head, target_ids, inv_temperature: float = 1.0,
                                   inv_temperature, _ptr(ws), ws.numel() * ws.element_size(), _stream())
     _check(rc, ctx)
     return logprob
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def tik_attn_decode_static(q, ctx_lens, k_cache, v_cache, block_table, max_ctx_len: int,
+                           softmax_scale: float, o: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                           dev_flags: Optional[torch.Tensor] = None) -> int:
+    """Decode attention through the entry point that allocates nothing: no library context,
+    no workspace (the scratch is a fixed array inside the library) and, unlike the other
+    wrappers, no output tensor is created here either - the caller passes `o`.  For callers
+    whose device memory is fully committed or who cannot afford cudaMalloc's synchronisation.
+    Returns the raw status code (0 = ok; -3 = the problem exceeds the fixed scratch)."""
+    bf = torch.bfloat16
+    B, Hq, d = q.shape
+    num_pages, Hkv, page, _ = k_cache.shape
+    return int(load().tik_attn_decode_static(
+        _ptr(q, bf), _ptr(o, bf), _ptr(lse, torch.float32), _ptr(ctx_lens, torch.int32),
+        _ptr(k_cache, bf), _ptr(v_cache, bf), _ptr(block_table, torch.int32), block_table.shape[1],
+        B, max_ctx_len, Hq, Hkv, d, page, num_pages, softmax_scale, _ptr(dev_flags, torch.int32),
+        _stream()))
