@@ -140,7 +140,7 @@ tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_he
  * GPU that loads the library until the process exits.  Meant for callers that cannot call
  * cudaMalloc: a server whose KV-cache pool already owns all free device memory, or a decode
  * loop that must avoid the device-wide synchronisation of cudaMalloc/cudaFree.
- *   - Needs B * Hq * ceil(max_ctx_len/2048) * (d+2) * 4 <= TIK_STATIC_SCRATCH_BYTES,
+ *   - Needs B * Hq * ceil(max_ctx_len/2048) * (d+4) * 4 <= TIK_STATIC_SCRATCH_BYTES,
  *     otherwise returns TIK_ERR_WORKSPACE and launches nothing.
  *   - Works on the current CUDA device.  The first call on each device resolves the
  *     scratch's device address and the driver's tensor-map encoder (host-side set-up, no

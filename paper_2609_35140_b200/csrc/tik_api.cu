@@ -124,7 +124,7 @@ size_t tik_workspace_bytes(int op, int64_t rows_or_batch, int Hq, int Hkv, int d
     if (op == TIK_OP_ATTN_DECODE) {
         if (rows_or_batch <= 0 || max_ctx <= 0) return 0;
         const int64_t nchunk = (max_ctx + CHUNK - 1) / CHUNK;
-        return static_cast<size_t>(rows_or_batch) * Hq * nchunk * (d + 2) * sizeof(float);
+        return static_cast<size_t>(rows_or_batch) * Hq * nchunk * (d + 4) * sizeof(float);
     }
     if (op == TIK_OP_TOKEN_LOGPROB) {
         if (rows_or_batch <= 0 || V <= 0) return 0;

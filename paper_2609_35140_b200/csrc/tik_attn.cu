@@ -5,9 +5,11 @@
 // One CTA owns one MMA tile of 128 query rows and walks 128-key KV tiles in ascending
 // order.  S = Q K^T and O += P V run on tcgen05 (M128 x N128 x K16 and M128 x Nd x K16,
 // fp32 accumulators in TMEM); Q, K, V arrive by TMA into 128B-swizzled shared memory
-// (K/V of the paged regimes are gathered page by page through the block table); the
-// online softmax is one thread per row, straight out of TMEM, with the arithmetic of
-// tik_core.cuh.  What differs between regimes is only where rows come from and where they
+// (K/V of the paged regimes are gathered page by page through the block table).  The CTA
+// is warp-specialised: one TMA warp, one MMA warp and two softmax warpgroups that each own
+// 64 of a tile's 128 key columns (and half of the O columns), working straight out of TMEM
+// with the arithmetic of tik_core.cuh; scores are double-buffered so the QK^T of tile j+1
+// runs under the softmax of tile j.  What differs between regimes is only where rows come from and where they
 // go:
 //   train   : rows = 128 consecutive tokens of one (sequence, query head); K/V packed
 //   prefill : same rows, aligned to absolute positions; K/V from pages
@@ -23,31 +25,37 @@ namespace tik {
 
 enum { MODE_TRAIN = 0, MODE_PREFILL = 1, MODE_DECODE = 2 };
 
+constexpr int ATTN_THREADS = 384;   // warp 0 TMA, warp 1 MMA, warps 2-3 idle, warps 4-11 softmax
+constexpr int KV_STAGES = 2;
+
 template <int D>
 struct AttnSmem {
     static constexpr uint32_t ATOM = 128 * 128;          // 128 rows x 64 bf16
     static constexpr uint32_t TILE = (D / 64) * ATOM;    // one Q, K or V tile
     static constexpr uint32_t OFF_Q = 0;
-    static constexpr uint32_t OFF_K = TILE;              // two stages
-    static constexpr uint32_t OFF_V = 3 * TILE;          // two stages
-    static constexpr uint32_t OFF_P = 5 * TILE;          // 128 rows x 128 keys bf16
-    static constexpr uint32_t OFF_BAR = OFF_P + 2 * ATOM;
-    static constexpr uint32_t BYTES = OFF_BAR + 128;
-    static constexpr uint32_t ALLOC = BYTES + 1024;      // slack for 1 KiB alignment
+    static constexpr uint32_t OFF_K = TILE;
+    static constexpr uint32_t OFF_V = OFF_K + KV_STAGES * TILE;
+    static constexpr uint32_t OFF_P = OFF_V + KV_STAGES * TILE;   // two buffers of 128 x 128 bf16
+    static constexpr uint32_t OFF_BAR = OFF_P + 2 * 2 * ATOM;
+    static constexpr uint32_t OFF_LX = OFF_BAR + 256;             // 2 x 128 floats: half row sums
+    static constexpr uint32_t BYTES = OFF_LX + 1024;
+    static constexpr uint32_t ALLOC = BYTES + 1024;               // slack for 1 KiB alignment
 };
 
 template <int D, int MODE>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
             const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
     using L = AttnSmem<D>;
     constexpr int NATOM = D / 64;
-    constexpr uint32_t TMEM_COLS = (D == 128) ? 512u : 256u;
-    constexpr uint32_t COL_S = 0, COL_OA = 128, COL_OB = 128 + D;
+    constexpr int DH = D / 2;                              // O columns owned by one softmax thread
+    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t COL_S = 0;                          // two score buffers of 128 columns
+    constexpr uint32_t COL_OA = 256, COL_OB = 256 + D;
     constexpr uint32_t IDESC_QK = mma_idesc_bf16(128, 128, false);
     constexpr uint32_t IDESC_PV = mma_idesc_bf16(128, D, true);
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---------------------------------------------------------------- work item
     int seq, head, kvh, T = 0, chunk = 0, ctx = 0, pos0 = 0;
@@ -107,33 +115,51 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const uint32_t sbase = raw_addr + pad;
     const uint32_t sQ = sbase + L::OFF_Q, sK = sbase + L::OFF_K, sV = sbase + L::OFF_V,
                    sP = sbase + L::OFF_P;
-    const uint32_t bar_q = sbase + L::OFF_BAR, bar_kv0 = bar_q + 8, bar_s = bar_q + 24,
-                   bar_o = bar_q + 32;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 40);
-    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 44);
+    // barriers (8 bytes each)
+    const uint32_t bar0 = sbase + L::OFF_BAR;
+    const uint32_t bar_q = bar0;                 // Q landed
+    const uint32_t bar_kfull = bar0 + 8;         // [KV_STAGES] K tile landed
+    const uint32_t bar_vfull = bar0 + 24;        // [KV_STAGES] V tile landed
+    const uint32_t bar_kempty = bar0 + 40;       // [KV_STAGES] QK^T that read the stage is done
+    const uint32_t bar_vempty = bar0 + 56;       // [KV_STAGES] PV that read the stage is done
+    const uint32_t bar_sfull = bar0 + 72;        // [2] scores ready in TMEM
+    const uint32_t bar_sempty = bar0 + 88;       // [2] softmax has read the scores (8 warps)
+    const uint32_t bar_pfull = bar0 + 104;       // [2] P written, O rescaled (8 warps)
+    const uint32_t bar_pempty = bar0 + 120;      // [2] PV done: P buffer free, O updated
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 136);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 140);
+    float* lx = reinterpret_cast<float*>(smem + L::OFF_LX);
 
     if (tid == 0) {
         mbar_init(bar_q, 1);
-        mbar_init(bar_kv0, 1);
-        mbar_init(bar_kv0 + 8, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
+        for (int i = 0; i < KV_STAGES; ++i) {
+            mbar_init(bar_kfull + 8 * i, 1);
+            mbar_init(bar_vfull + 8 * i, 1);
+            mbar_init(bar_kempty + 8 * i, 1);
+            mbar_init(bar_vempty + 8 * i, 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_sfull + 8 * i, 1);
+            mbar_init(bar_sempty + 8 * i, 8);
+            mbar_init(bar_pfull + 8 * i, 8);
+            mbar_init(bar_pempty + 8 * i, 1);
+        }
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmQ);
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmV);
     }
-    if (warp == 0) {
+    if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
         tmem_relinquish();
     }
     if (MODE == MODE_DECODE) {
-        // rows >= G of the Q tile are never loaded: make them zero; P rows of idle warps too
-        uint4 z = make_uint4(0, 0, 0, 0);
-        for (uint32_t i = tid; i < L::TILE / 16; i += 128)
+        // rows >= G of the Q tile are never loaded and P rows of idle warps never written: zero them
+        const uint4 z = make_uint4(0, 0, 0, 0);
+        for (uint32_t i = tid; i < L::TILE / 16; i += ATTN_THREADS)
             reinterpret_cast<uint4*>(smem + L::OFF_Q)[i] = z;
-        for (uint32_t i = tid; i < 2 * L::ATOM / 16; i += 128)
+        for (uint32_t i = tid; i < 4 * L::ATOM / 16; i += ATTN_THREADS)
             reinterpret_cast<uint4*>(smem + L::OFF_P)[i] = z;
         fence_proxy_async_smem();
     }
@@ -141,252 +167,321 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tlane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
 
-    // ---------------------------------------------------------------- loaders (thread 0)
-    auto load_q = [&]() {
-        if (MODE == MODE_DECODE) {
-            mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
-            for (int a = 0; a < NATOM; ++a)
-                tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
-        } else {
-            mbar_expect_tx(bar_q, L::TILE);
-            for (int a = 0; a < NATOM; ++a)
-                tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
-        }
+    auto chunk_of = [&](int it) { return (tile_first + it) / TILES_PER_CHUNK; };
+    auto is_chunk_start = [&](int it) { return ((tile_first + it) % TILES_PER_CHUNK) == 0; };
+    auto col_o_of = [&](int it) -> uint32_t {
+        return (MODE == MODE_DECODE || chunk_of(it) == 0) ? COL_OA : COL_OB;
     };
-    auto load_kv = [&](int j, int st) {
-        const uint32_t bar = bar_kv0 + 8 * st;
-        const uint32_t dK = sK + st * L::TILE, dV = sV + st * L::TILE;
-        mbar_expect_tx(bar, 2 * L::TILE);
-        if (MODE == MODE_TRAIN) {
-            const int row = static_cast<int>(tok0) + 128 * j;
-            for (int a = 0; a < NATOM; ++a) {
-                tma_load_3d(dK + a * L::ATOM, &tmK, bar, a * 64, kvh, row);
-                tma_load_3d(dV + a * L::ATOM, &tmV, bar, a * 64, kvh, row);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            if (MODE == MODE_DECODE) {
+                mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
+                for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
+            } else {
+                mbar_expect_tx(bar_q, L::TILE);
+                for (int a = 0; a < NATOM; ++a)
+                    tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
             }
-        } else {
-            const int lp0 = (128 * j) / p.page_size;
-            for (int i = 0; i < p.pages_per_tile; ++i) {
-                const int lp = lp0 + i;
-                int phys = p.num_pages;   // out of range: the box is filled with zeros
-                if (lp * p.page_size < ctx) {
-                    if (lp < p.max_blocks) phys = p.block_table[static_cast<long long>(seq) * p.max_blocks + lp];
-                    else phys = -1;
-                    if (phys < 0 || phys >= p.num_pages) {
-                        atomicOr(p.dev_status, TIK_DEV_BAD_BLOCK);
-                        phys = p.num_pages;
+            for (int it = 0; it < n_tiles; ++it) {
+                const int j = tile_first + it;
+                const int st = it % KV_STAGES;
+                const uint32_t use = it / KV_STAGES;
+                const uint32_t dK = sK + st * L::TILE, dV = sV + st * L::TILE;
+                int phys[8];
+                if (MODE != MODE_TRAIN) {
+                    const int lp0 = (128 * j) / p.page_size;
+                    for (int i = 0; i < p.pages_per_tile; ++i) {
+                        const int lp = lp0 + i;
+                        int ph = p.num_pages;   // out of range: the box is filled with zeros
+                        if (lp * p.page_size < ctx) {
+                            ph = (lp < p.max_blocks) ? p.block_table[static_cast<long long>(seq) * p.max_blocks + lp] : -1;
+                            if (ph < 0 || ph >= p.num_pages) {
+                                atomicOr(p.dev_status, TIK_DEV_BAD_BLOCK);
+                                ph = p.num_pages;
+                            }
+                        }
+                        phys[i] = ph;
                     }
                 }
-                const uint32_t off = static_cast<uint32_t>(i * p.page_size) * 128u;
-                for (int a = 0; a < NATOM; ++a) {
-                    tma_load_4d(dK + a * L::ATOM + off, &tmK, bar, a * 64, 0, kvh, phys);
-                    tma_load_4d(dV + a * L::ATOM + off, &tmV, bar, a * 64, 0, kvh, phys);
+                for (int kv = 0; kv < 2; ++kv) {
+                    const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
+                    const uint32_t empty = (kv ? bar_vempty : bar_kempty) + 8 * st;
+                    const uint32_t dst = kv ? dV : dK;
+                    const CUtensorMap* tm = kv ? &tmV : &tmK;
+                    if (use > 0) mbar_wait(empty, (use - 1) & 1, abort_word, p.dev_status);
+                    mbar_expect_tx(full, L::TILE);
+                    if (MODE == MODE_TRAIN) {
+                        const int row = static_cast<int>(tok0) + 128 * j;
+                        for (int a = 0; a < NATOM; ++a) tma_load_3d(dst + a * L::ATOM, tm, full, a * 64, kvh, row);
+                    } else {
+                        for (int i = 0; i < p.pages_per_tile; ++i) {
+                            const uint32_t off = static_cast<uint32_t>(i * p.page_size) * 128u;
+                            for (int a = 0; a < NATOM; ++a)
+                                tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, phys[i]);
+                        }
+                    }
                 }
             }
         }
-    };
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            auto issue_qk = [&](int x) {
+                const int st = x % KV_STAGES, b = x & 1;
+                mbar_wait(bar_kfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
+                if (x >= 2) mbar_wait(bar_sempty + 8 * b, ((x >> 1) - 1) & 1, abort_word, p.dev_status);
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t koff = (ks >> 2) * L::ATOM + (ks & 3) * 32;
+                    mma_ss(tmem + COL_S + 128 * b, smem_desc_sw128(sQ + koff, 0, 1024),
+                           smem_desc_sw128(sK + st * L::TILE + koff, 0, 1024), IDESC_QK, ks > 0);
+                }
+                mma_commit(bar_sfull + 8 * b);
+                mma_commit(bar_kempty + 8 * st);
+            };
+            auto issue_pv = [&](int x) {
+                const int st = x % KV_STAGES, b = x & 1;
+                mbar_wait(bar_vfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
+                mbar_wait(bar_pfull + 8 * b, (x >> 1) & 1, abort_word, p.dev_status);
+                tc_fence_after();
+                const uint32_t col_o = col_o_of(x);
+                const bool fresh = is_chunk_start(x);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t poff = b * 2 * L::ATOM + (ks >> 2) * L::ATOM + (ks & 3) * 32;
+                    mma_ss(tmem + col_o, smem_desc_sw128(sP + poff, 0, 1024),
+                           smem_desc_sw128(sV + st * L::TILE + ks * 2048, L::ATOM, 1024), IDESC_PV,
+                           (fresh && ks == 0) ? 0u : 1u);
+                }
+                mma_commit(bar_vempty + 8 * st);
+                mma_commit(bar_pempty + 8 * b);
+            };
+            mbar_wait(bar_q, 0, abort_word, p.dev_status);
+            issue_qk(0);
+            for (int it = 0; it < n_tiles; ++it) {
+                if (it + 1 < n_tiles) issue_qk(it + 1);
+                issue_pv(it);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ softmax (two warpgroups)
+        const int wg = (warp - 4) >> 2;                     // owns key columns [64 wg, 64 wg + 64)
+        const int quarter = warp & 3;                       // TMEM lane quarter of this warp
+        const int r = quarter * 32 + lane;                  // tile row == TMEM lane
+        const uint32_t tlane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+        const int qpos = (MODE == MODE_DECODE) ? (ctx - 1) : (128 * T + r);
+        const bool active = (MODE != MODE_DECODE) || (quarter == 0);
+        const float c = p.c;
+        float m_run = -CUDART_INF_F, l_run = 0.0f;          // current chunk (l: this thread's half)
+        float m_prev = 0.0f, l_prev = 0.0f;                  // finished chunk waiting to be folded
+        float M_g = -CUDART_INF_F, L_g = 0.0f;               // folded state of earlier chunks
+        bool fold_pending = false;
+        int prev_chunk = 0;
 
-    if (tid == 0) {
-        load_q();
-        load_kv(tile_first, 0);
-    }
-
-    // ---------------------------------------------------------------- per-row state
-    const int r = tid;                                      // tile row == TMEM lane
-    const int qpos = (MODE == MODE_DECODE) ? (ctx - 1) : (128 * T + r);
-    const bool softmax_active = (MODE != MODE_DECODE) || (warp == 0);
-    const float c = p.c;
-    float m_run = -CUDART_INF_F, l_run = 0.0f;              // state of the current chunk
-    float M_g = -CUDART_INF_F, L_g = 0.0f;                  // folded state of earlier chunks
-    uint32_t par_s = 0, par_o = 0, par_kv[2] = {0, 0};
-    uint32_t col_o = COL_OA;                                // chunk 0 accumulates in place
-
-    for (int it = 0; it < n_tiles; ++it) {
-        const int j = tile_first + it;
-        const int st = it & 1;
-        const bool chunk_start = (j % TILES_PER_CHUNK) == 0;
-        const bool chunk_end = ((j % TILES_PER_CHUNK) == TILES_PER_CHUNK - 1) || (it == n_tiles - 1);
-        const int chunk_idx = j / TILES_PER_CHUNK;
-        if (MODE != MODE_DECODE && chunk_start) col_o = (chunk_idx == 0) ? COL_OA : COL_OB;
-
-        if (tid == 0) {
-            if (it + 1 < n_tiles) load_kv(j + 1, st ^ 1);
-            if (it == 0) mbar_wait(bar_q, 0, abort_word, p.dev_status);
-            mbar_wait(bar_kv0 + 8 * st, par_kv[st], abort_word, p.dev_status);
+        // waits until the PV of tile `x` has completed (O and the P buffer are consistent)
+        auto wait_pv = [&](int x) {
+            mbar_wait(bar_pempty + 8 * (x & 1), (x >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
+        };
+        // folds the finished chunk (m_prev, l_prev, O_B) into the global state; PV must be done
+        auto fold_chunk = [&]() {
+            if (prev_chunk == 0) {           // chunk 0 accumulated in place in O_A
+                M_g = m_prev;
+                L_g = l_prev;
+            } else {
+                const FoldCoef f = fold_coef(M_g, m_prev, c);
+                L_g = fold_value(L_g, l_prev, f);
+                M_g = f.M_new;
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t koff = (ks >> 2) * L::ATOM + (ks & 3) * 32;
-                mma_ss(tmem + COL_S, smem_desc_sw128(sQ + koff, 0, 1024),
-                       smem_desc_sw128(sK + st * L::TILE + koff, 0, 1024), IDESC_QK, ks > 0);
-            }
-            mma_commit(bar_s);
-        }
-        par_kv[st] ^= 1;
-        mbar_wait(bar_s, par_s, abort_word, p.dev_status);
-        par_s ^= 1;
-        tc_fence_after();
-
-        if (softmax_active) {
-            const int kmax = qpos - 128 * j;      // columns > kmax are masked
-            // pass 1: tile maximum
-            float mt = -CUDART_INF_F;
+                for (int cc = 0; cc < DH / 32; ++cc) {
+                    uint32_t a[32], b[32];
+                    tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, a);
+                    tmem_ld32(tlane + COL_OB + DH * wg + 32 * cc, b);
+                    tmem_wait_ld();
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t v[32];
-                tmem_ld32(tlane + COL_S + 32 * cc, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float s = __uint_as_float(v[i]);
-                    if (32 * cc + i > kmax) s = -CUDART_INF_F;
-                    mt = fmaxf(mt, s);
+                    for (int i = 0; i < 32; ++i)
+                        a[i] = __float_as_uint(fold_value(__uint_as_float(a[i]), __uint_as_float(b[i]), f));
+                    tmem_st32(tlane + COL_OA + DH * wg + 32 * cc, a);
                 }
+                tmem_wait_st();
             }
-            const float m_new = fmaxf(m_run, mt);
-            const float neg_mc = -__fmul_rn(m_new, c);
-            const float alpha = softmax_alpha(m_run, m_new, c);
-            // pass 2: p, row sum, bf16 P into swizzled shared memory
-            RowSum8 rs;
-            rs.reset();
+        };
+
+        for (int it = 0; it < n_tiles; ++it) {
+            const int j = tile_first + it;
+            const int b = it & 1;
+            const bool chunk_start = is_chunk_start(it);
+            if (MODE != MODE_DECODE && chunk_start && it > 0) {
+                m_prev = m_run;
+                l_prev = l_run;
+                prev_chunk = chunk_of(it - 1);
+                fold_pending = true;
+                m_run = -CUDART_INF_F;
+                l_run = 0.0f;
+            }
+            mbar_wait(bar_sfull + 8 * b, (it >> 1) & 1, abort_word, p.dev_status);
+            tc_fence_after();
+            uint32_t pk[32];
+            float alpha = 1.0f;
+            if (active) {
+                const int kmax = qpos - 128 * j;            // columns > kmax are masked
+                const uint32_t ts = tlane + COL_S + 128 * b;
+                uint32_t own[64];
+                float mt = -CUDART_INF_F;
+                {   // the other half only contributes to the row maximum
+                    uint32_t oth[32];
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t v[32];
-                tmem_ld32(tlane + COL_S + 32 * cc, v);
-                tmem_wait_ld();
-                uint32_t pk[16];
+                    for (int cc = 0; cc < 2; ++cc) {
+                        tmem_ld32(ts + 64 * (wg ^ 1) + 32 * cc, oth);
+                        if (cc == 0) {
+                            tmem_ld32(ts + 64 * wg, *reinterpret_cast<uint32_t(*)[32]>(&own[0]));
+                            tmem_ld32(ts + 64 * wg + 32, *reinterpret_cast<uint32_t(*)[32]>(&own[32]));
+                        }
+                        tmem_wait_ld();
+                        const int col0 = 64 * (wg ^ 1) + 32 * cc;
+                        if (kmax >= 127) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float p0 = softmax_p(__uint_as_float(v[i]), c, neg_mc);
-                    float p1 = softmax_p(__uint_as_float(v[i + 1]), c, neg_mc);
-                    if (32 * cc + i > kmax) p0 = 0.0f;
-                    if (32 * cc + i + 1 > kmax) p1 = 0.0f;
-                    rowsum_add(rs, 32 * cc + i, p0);
-                    rowsum_add(rs, 32 * cc + i + 1, p1);
+                            for (int i = 0; i < 32; ++i) mt = fmaxf(mt, __uint_as_float(oth[i]));
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                mt = fmaxf(mt, (col0 + i > kmax) ? -CUDART_INF_F : __uint_as_float(oth[i]));
+                        }
+                    }
+                }
+                const int own0 = 64 * wg;
+                if (kmax < 127) {
+#pragma unroll
+                    for (int i = 0; i < 64; ++i)
+                        if (own0 + i > kmax) own[i] = 0xff800000u;      // -inf
+                }
+#pragma unroll
+                for (int i = 0; i < 64; ++i) mt = fmaxf(mt, __uint_as_float(own[i]));
+                const float m_new = fmaxf(m_run, mt);
+                const float neg_mc = -__fmul_rn(m_new, c);
+                alpha = softmax_alpha(m_run, m_new, c);
+                RowSum4 rs;
+                rs.reset();
+#pragma unroll
+                for (int i = 0; i < 64; i += 2) {
+                    // a masked score is -inf: fma gives -inf and ex2 gives +0 exactly
+                    const float p0 = softmax_p(__uint_as_float(own[i]), c, neg_mc);
+                    const float p1 = softmax_p(__uint_as_float(own[i + 1]), c, neg_mc);
+                    rowsum_add(rs, i, p0);
+                    rowsum_add(rs, i + 1, p1);
                     pk[i >> 1] = pack_bf16x2(p0, p1);
                 }
+                l_run = __fmaf_rn(l_run, alpha, rs.total());
+                m_run = m_new;
+            }
+            // scores of this tile are in registers: release the TMEM buffer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_sempty + 8 * b);
+            // the P buffer was last read by the PV of tile it-2
+            if (it >= 2) wait_pv(it - 2);
+            if (active) {
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int chunk16 = 4 * (cc & 1) + q4;      // 16-byte chunk within the 128 B row
-                    const uint32_t off = L::OFF_P + (cc >> 1) * L::ATOM + r * 128 +
-                                         ((chunk16 ^ (r & 7)) << 4);
+                for (int q4 = 0; q4 < 8; ++q4) {
+                    const uint32_t off = L::OFF_P + (b * 2 + wg) * L::ATOM + r * 128 + ((q4 ^ (r & 7)) << 4);
                     *reinterpret_cast<uint4*>(smem + off) =
                         make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
                 }
+                fence_proxy_async_smem();
             }
-            l_run = __fmaf_rn(l_run, alpha, rs.total());
-            m_run = m_new;
-            // rescale the chunk accumulator (not on the first tile of a chunk, which overwrites)
-            if (!chunk_start && !__all_sync(0xffffffffu, alpha == 1.0f)) {
+            if (fold_pending) {                       // uniform over the CTA
+                wait_pv(it - 1);
+                if (active) fold_chunk();
+                fold_pending = false;
+            } else if (!chunk_start && active && !__all_sync(0xffffffffu, alpha == 1.0f)) {
+                // rescale this thread's half of the chunk accumulator
+                wait_pv(it - 1);
+                const uint32_t to = tlane + col_o_of(it) + DH * wg;
 #pragma unroll
-                for (int cc = 0; cc < D / 32; ++cc) {
+                for (int cc = 0; cc < DH / 32; ++cc) {
                     uint32_t v[32];
-                    tmem_ld32(tlane + col_o + 32 * cc, v);
+                    tmem_ld32(to + 32 * cc, v);
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
                         v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
-                    tmem_st32(tlane + col_o + 32 * cc, v);
+                    tmem_st32(to + 32 * cc, v);
                 }
                 tmem_wait_st();
             }
-            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_pfull + 8 * b);
         }
-        tc_fence_before();
-        __syncthreads();
 
-        if (tid == 0) {
-            tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                const uint32_t poff = (ks >> 2) * L::ATOM + (ks & 3) * 32;
-                mma_ss(tmem + col_o, smem_desc_sw128(sP + poff, 0, 1024),
-                       smem_desc_sw128(sV + st * L::TILE + ks * 2048, L::ATOM, 1024), IDESC_PV,
-                       (chunk_start && ks == 0) ? 0u : 1u);
-            }
-            mma_commit(bar_o);
-        }
-        mbar_wait(bar_o, par_o, abort_word, p.dev_status);
-        par_o ^= 1;
-        tc_fence_after();
-
-        if (chunk_end) {
-            if (MODE == MODE_DECODE) {
-                if (warp == 0 && r < p.G) {
-                    const long long slot =
-                        (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk;
-                    p.part_ml[2 * slot] = m_run;
-                    p.part_ml[2 * slot + 1] = l_run;
-                }
-                if (warp == 0) {
-#pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
-                        uint32_t v[32];
-                        tmem_ld32(tlane + col_o + 32 * cc, v);
-                        tmem_wait_ld();
-                        if (r < p.G) {
-                            const long long slot =
-                                (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk;
-                            float4* dst = reinterpret_cast<float4*>(p.part_o + slot * D + 32 * cc);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                                     __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-                        }
-                    }
-                }
-            } else {
-                if (chunk_idx == 0) {
-                    M_g = m_run;
-                    L_g = l_run;
+        // ---- all tiles issued: wait for the last PV, then finish the row
+        wait_pv(n_tiles - 1);
+        if (MODE == MODE_DECODE) {
+            if (active && r < p.G) {
+                const long long slot = (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk;
+                if (wg == 0) {
+                    p.part_ml[4 * slot] = m_run;
+                    p.part_ml[4 * slot + 1] = l_run;
                 } else {
-                    const FoldCoef f = fold_coef(M_g, m_run, c);
-                    L_g = fold_value(L_g, l_run, f);
-                    M_g = f.M_new;
-#pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
-                        uint32_t a[32], b[32];
-                        tmem_ld32(tlane + COL_OA + 32 * cc, a);
-                        tmem_ld32(tlane + COL_OB + 32 * cc, b);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            a[i] = __float_as_uint(fold_value(__uint_as_float(a[i]), __uint_as_float(b[i]), f));
-                        tmem_st32(tlane + COL_OA + 32 * cc, a);
-                    }
-                    tmem_wait_st();
+                    p.part_ml[4 * slot + 2] = l_run;
                 }
-                m_run = -CUDART_INF_F;
-                l_run = 0.0f;
             }
-        }
-    }
-
-    // ---------------------------------------------------------------- finalise (train / prefill)
-    if (MODE != MODE_DECODE) {
-        const float inv = finalize_inv(L_g);
-        const bool valid = (r >= row_lo) && (r < row_hi);
-        const long long orow = (qrow0 + r) * p.Hq + head;
-        __nv_bfloat16* optr = reinterpret_cast<__nv_bfloat16*>(p.o) + orow * D;
+            if (active) {
 #pragma unroll
-        for (int cc = 0; cc < D / 32; ++cc) {
-            uint32_t v[32];
-            tmem_ld32(tlane + COL_OA + 32 * cc, v);
-            tmem_wait_ld();
-            if (valid) {
-                uint32_t pk[16];
+                for (int cc = 0; cc < DH / 32; ++cc) {
+                    uint32_t v[32];
+                    tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, v);
+                    tmem_wait_ld();
+                    if (r < p.G) {
+                        const long long slot =
+                            (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk;
+                        float4* dst = reinterpret_cast<float4*>(p.part_o + slot * D + DH * wg + 32 * cc);
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    pk[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv),
-                                        finalize_o(__uint_as_float(v[2 * i + 1]), inv));
-                uint4* dst = reinterpret_cast<uint4*>(optr + 32 * cc);
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                        for (int i = 0; i < 8; ++i)
+                            dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                                 __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                    }
+                }
             }
+        } else {
+            m_prev = m_run;
+            l_prev = l_run;
+            prev_chunk = chunk_of(n_tiles - 1);
+            fold_chunk();
+            // exchange the half row sums between the two threads of a row
+            lx[wg * 128 + r] = L_g;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            const float l_lo = lx[r], l_hi = lx[128 + r];
+            const float Ltot = finalize_l(l_lo, l_hi);
+            const float inv = finalize_inv(Ltot);
+            const bool valid = (r >= row_lo) && (r < row_hi);
+            const long long orow = (qrow0 + r) * p.Hq + head;
+            __nv_bfloat16* optr = reinterpret_cast<__nv_bfloat16*>(p.o) + orow * D + DH * wg;
+#pragma unroll
+            for (int cc = 0; cc < DH / 32; ++cc) {
+                uint32_t v[32];
+                tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, v);
+                tmem_wait_ld();
+                if (valid) {
+                    uint32_t o16[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        o16[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv),
+                                             finalize_o(__uint_as_float(v[2 * i + 1]), inv));
+                    uint4* dst = reinterpret_cast<uint4*>(optr + 32 * cc);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        dst[i] = make_uint4(o16[4 * i], o16[4 * i + 1], o16[4 * i + 2], o16[4 * i + 3]);
+                }
+            }
+            if (valid && wg == 0 && p.lse) p.lse[orow] = finalize_lse(M_g, Ltot, c);
         }
-        if (valid && p.lse) p.lse[orow] = finalize_lse(M_g, L_g, c);
     }
 
     // ---------------------------------------------------------------- teardown
@@ -397,12 +492,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
+    if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
 // ------------------------------------------------------------------ split-KV combine
 // One block per (sequence, query head), one thread per head_dim column; folds the chunk
-// partials in ascending chunk order and normalises.
+// partials (m, l_lo, l_hi, O) in ascending chunk order and normalises.
 template <int D>
 __global__ void __launch_bounds__(D) combine_kernel(const AttnParams p) {
     const int b = blockIdx.x / p.Hq;
@@ -411,20 +506,22 @@ __global__ void __launch_bounds__(D) combine_kernel(const AttnParams p) {
     const int nc = (ctx + CHUNK - 1) / CHUNK;
     const long long slot0 = static_cast<long long>(blockIdx.x) * p.nchunk_max;
     const int col = threadIdx.x;
-    float M = p.part_ml[2 * slot0], Lsum = p.part_ml[2 * slot0 + 1];
+    float M = p.part_ml[4 * slot0], L_lo = p.part_ml[4 * slot0 + 1], L_hi = p.part_ml[4 * slot0 + 2];
     float O = p.part_o[slot0 * D + col];
     for (int ch = 1; ch < nc; ++ch) {
-        const float m_c = p.part_ml[2 * (slot0 + ch)], l_c = p.part_ml[2 * (slot0 + ch) + 1];
+        const float* ml = p.part_ml + 4 * (slot0 + ch);
         const float o_c = p.part_o[(slot0 + ch) * D + col];
-        const FoldCoef f = fold_coef(M, m_c, p.c);
-        Lsum = fold_value(Lsum, l_c, f);
+        const FoldCoef f = fold_coef(M, ml[0], p.c);
+        L_lo = fold_value(L_lo, ml[1], f);
+        L_hi = fold_value(L_hi, ml[2], f);
         O = fold_value(O, o_c, f);
         M = f.M_new;
     }
-    const float inv = finalize_inv(Lsum);
+    const float Ltot = finalize_l(L_lo, L_hi);
+    const float inv = finalize_inv(Ltot);
     reinterpret_cast<__nv_bfloat16*>(p.o)[static_cast<long long>(blockIdx.x) * D + col] =
         __float2bfloat16_rn(finalize_o(O, inv));
-    if (p.lse && col == 0) p.lse[blockIdx.x] = finalize_lse(M, Lsum, p.c);
+    if (p.lse && col == 0) p.lse[blockIdx.x] = finalize_lse(M, Ltot, p.c);
 }
 
 // ------------------------------------------------------------------ KV-cache write
@@ -474,7 +571,7 @@ static cudaError_t launch_attn_t(dim3 grid, const CUtensorMap& tmQ, const CUtens
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, 128, AttnSmem<D>::ALLOC, stream>>>(tmQ, tmK, tmV, p);
+    kern<<<grid, ATTN_THREADS, AttnSmem<D>::ALLOC, stream>>>(tmQ, tmK, tmV, p);
     return cudaGetLastError();
 }
 

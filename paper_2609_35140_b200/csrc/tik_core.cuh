@@ -17,11 +17,11 @@
 //   * Mask: select -inf where key position > query position (no arithmetic on masked
 //     scores, so masked K contents never matter).
 //   * Per tile and row: m' = max(m, tile max); p = ex2.approx.ftz(fma(s, c, -(m' * c)));
-//     row sum in the fixed 8-chain shape below; alpha = ex2.approx.ftz((m - m') * c);
-//     l = fma(l, alpha, rowsum); O = O * alpha with a non-flushing IEEE multiply (so
+//     row sums in the fixed two-halves-of-four-chains shape below; alpha = ex2.approx.ftz((m - m') * c);
+//     l_half = fma(l_half, alpha, rowsum of that 64-column half); O = O * alpha with a non-flushing IEEE multiply (so
 //     skipping it when alpha == 1.0f is bit-neutral); P rounded to bf16 (RNE) for the PV
 //     MMA while l sums the unrounded fp32 p.
-//   * Finalise: o = O * rcp.rn(l), rounded to bf16 (RNE).
+//   * Finalise: l = l_lo + l_hi; o = O * rcp.rn(l), rounded to bf16 (RNE).
 #pragma once
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -38,7 +38,7 @@ constexpr float LN2_F = 0.69314718055994530942f;
 constexpr int LP_TILE = 128;          // vocabulary columns per log-sum-exp tile
 constexpr int LP_SUPER = 1024;        // vocabulary columns per super-chunk (8 tiles)
 
-#define TIK_CONTRACT_ID "tik1-BN128-CH2048-M128N128K16-ex2ftz-sum8-LP128x1024"
+#define TIK_CONTRACT_ID "tik2-BN128-CH2048-M128N128K16-ex2ftz-sum2x4-LP128x1024"
 
 __device__ __forceinline__ float ex2_ftz(float x) {
     float y;
@@ -46,27 +46,39 @@ __device__ __forceinline__ float ex2_ftz(float x) {
     return y;
 }
 
-// Running row sum in a fixed shape: chain index = 4 * (col / 64) + ((col / 2) % 4); every
-// chain adds its columns in ascending order; the eight chains are combined as
-// ((a0+a1)+(a2+a3)) + ((a4+a5)+(a6+a7)).  The shape lets a row be summed by one thread,
-// by two threads owning 64 columns each, or by four threads owning interleaved column
-// pairs, with identical bits.
-struct RowSum8 {
-    float a[8];
+// Row sums have a fixed shape.  The 128 columns of a tile are two halves of 64; within a
+// half, chain k adds the columns with (col / 2) % 4 == k in ascending order and the four
+// chains are combined as (a0+a1)+(a2+a3).  Attention keeps the two halves apart for the
+// whole computation: every row carries (l_lo, l_hi), each updated as l = fma(l, alpha, half
+// sum), folded across chunks separately, and added only once, right before the final
+// reciprocal.  So a row can be summed by one thread, by two threads owning 64 columns each,
+// or by four threads owning interleaved column pairs, with identical bits.
+struct RowSum4 {
+    float a[4];
     __device__ __forceinline__ void reset() {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) a[i] = 0.0f;
+        for (int i = 0; i < 4; ++i) a[i] = 0.0f;
     }
     __device__ __forceinline__ float total() const {
-        const float lo = __fadd_rn(__fadd_rn(a[0], a[1]), __fadd_rn(a[2], a[3]));
-        const float hi = __fadd_rn(__fadd_rn(a[4], a[5]), __fadd_rn(a[6], a[7]));
-        return __fadd_rn(lo, hi);
+        return __fadd_rn(__fadd_rn(a[0], a[1]), __fadd_rn(a[2], a[3]));
     }
 };
-// `col` must be a compile-time constant after unrolling.
-__device__ __forceinline__ void rowsum_add(RowSum8& s, int col, float p) {
-    const int chain = ((col >> 6) << 2) | ((col >> 1) & 3);
+// `col` (0..63 within the half) must be a compile-time constant after unrolling.
+__device__ __forceinline__ void rowsum_add(RowSum4& s, int col, float p) {
+    const int chain = (col >> 1) & 3;
     s.a[chain] = __fadd_rn(s.a[chain], p);
+}
+// The log-probability kernels sum a 128-column tile as half(0..63) + half(64..127).
+struct RowSum8 {
+    RowSum4 h[2];
+    __device__ __forceinline__ void reset() {
+        h[0].reset();
+        h[1].reset();
+    }
+    __device__ __forceinline__ float total() const { return __fadd_rn(h[0].total(), h[1].total()); }
+};
+__device__ __forceinline__ void rowsum_add(RowSum8& s, int col, float p) {
+    rowsum_add(s.h[col >> 6], col & 63, p);
 }
 
 // exponent argument of one score: s * c - mc, one fused multiply-add.
@@ -101,6 +113,7 @@ __device__ __forceinline__ float fold_value(float X, float x_c, const FoldCoef& 
     return __fmaf_rn(X, f.A, __fmul_rn(x_c, f.B));
 }
 
+__device__ __forceinline__ float finalize_l(float l_lo, float l_hi) { return __fadd_rn(l_lo, l_hi); }
 __device__ __forceinline__ float finalize_inv(float L) { return __frcp_rn(L); }
 __device__ __forceinline__ float finalize_o(float O, float inv) { return __fmul_rn(O, inv); }
 // natural-log log-sum-exp of the scaled scores: (M * c + log2 L) * ln 2

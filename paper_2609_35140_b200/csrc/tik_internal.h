@@ -33,7 +33,7 @@ struct AttnParams {
     int page_size, pages_per_tile, num_pages;
     float c;                     // softmax_scale * log2(e)
     float* part_o;               // decode: [B][Hq][nchunk_max][d]
-    float* part_ml;              // decode: [B][Hq][nchunk_max][2]
+    float* part_ml;              // decode: [B][Hq][nchunk_max][4] = m, l_lo, l_hi, unused
     int nchunk_max;
     int* dev_status;
 };

@@ -30,12 +30,12 @@ def test_library_exports_every_declared_symbol():
 
 def test_host_only_calls_work_without_a_gpu():
     from paper_2609_35140_b200 import binding
-    assert binding.contract_id().startswith("tik1-")
+    assert binding.contract_id().startswith("tik")
     lib = binding.load()
     assert lib.tik_status_str(0) == b"ok"
     assert lib.tik_status_str(-3) == b"workspace too small"
-    # decode scratch: B * Hq * chunks * (d + 2) floats; log-prob: T * (2 * super-chunks + 1) floats
-    assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 16384) == 16 * 32 * 8 * 130 * 4
-    assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 2049) == 16 * 32 * 2 * 130 * 4
+    # decode scratch: B * Hq * chunks * (d + 4) floats; log-prob: T * (2 * super-chunks + 1) floats
+    assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 16384) == 16 * 32 * 8 * 132 * 4
+    assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 2049) == 16 * 32 * 2 * 132 * 4
     assert binding.workspace_bytes(binding.OP_TOKEN_LOGPROB, 1000, H=4096, V=151936) == 1000 * (2 * 149 + 1) * 4
     assert binding.workspace_bytes(binding.OP_ATTN_TRAIN_FWD, 1000, 8, 2, 128, 4096) == 0

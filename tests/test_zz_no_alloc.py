@@ -63,8 +63,8 @@ def test_static_decode_refuses_problems_beyond_its_scratch():
     tik.load()
     w, q, ctx, kc, vc, bt = _case(tik, [64, 64], [10, 20], 8, 2, 128, 64, 203)
     out = torch.full((2, 8, 128), 7.0, dtype=torch.bfloat16, device="cuda")
-    # claim a context so long that 2 * 8 * chunks * 130 * 4 bytes exceeds the fixed scratch
-    huge_ctx = 2048 * (tik.STATIC_SCRATCH_BYTES // (2 * 8 * 130 * 4) + 1)
+    # claim a context so long that 2 * 8 * chunks * 132 * 4 bytes exceeds the fixed scratch
+    huge_ctx = 2048 * (tik.STATIC_SCRATCH_BYTES // (2 * 8 * 132 * 4) + 1)
     rc = tik.tik_attn_decode_static(q, ctx, kc, vc, bt, huge_ctx, w.softmax_scale, out)
     assert rc == -3
     torch.cuda.synchronize()
