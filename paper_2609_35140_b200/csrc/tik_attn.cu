@@ -25,8 +25,8 @@ namespace tik {
 
 enum { MODE_TRAIN = 0, MODE_PREFILL = 1, MODE_DECODE = 2 };
 
-constexpr int ATTN_THREADS = 384;   // warp 0 TMA, warp 1 MMA, warps 2-3 idle, warps 4-11 softmax
-constexpr int KV_STAGES = 2;
+constexpr int ATTN_THREADS = 384;   // warp 0 TMA (Q, K), warp 1 MMA, warp 2 TMA (V), warp 3 idle, warps 4-11 softmax
+constexpr int KV_STAGES = 3;
 
 template <int D>
 struct AttnSmem {
@@ -35,8 +35,7 @@ struct AttnSmem {
     static constexpr uint32_t OFF_Q = 0;
     static constexpr uint32_t OFF_K = TILE;
     static constexpr uint32_t OFF_V = OFF_K + KV_STAGES * TILE;
-    static constexpr uint32_t OFF_P = OFF_V + KV_STAGES * TILE;   // two buffers of 128 x 128 bf16
-    static constexpr uint32_t OFF_BAR = OFF_P + 2 * 2 * ATOM;
+    static constexpr uint32_t OFF_BAR = OFF_V + KV_STAGES * TILE;
     static constexpr uint32_t OFF_LX = OFF_BAR + 256;             // 2 x 128 floats: half row sums
     static constexpr uint32_t BYTES = OFF_LX + 1024;
     static constexpr uint32_t ALLOC = BYTES + 1024;               // slack for 1 KiB alignment
@@ -113,21 +112,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
     uint8_t* smem = smem_raw + pad;
     const uint32_t sbase = raw_addr + pad;
-    const uint32_t sQ = sbase + L::OFF_Q, sK = sbase + L::OFF_K, sV = sbase + L::OFF_V,
-                   sP = sbase + L::OFF_P;
+    const uint32_t sQ = sbase + L::OFF_Q, sK = sbase + L::OFF_K, sV = sbase + L::OFF_V;
     // barriers (8 bytes each)
     const uint32_t bar0 = sbase + L::OFF_BAR;
     const uint32_t bar_q = bar0;                 // Q landed
     const uint32_t bar_kfull = bar0 + 8;         // [KV_STAGES] K tile landed
-    const uint32_t bar_vfull = bar0 + 24;        // [KV_STAGES] V tile landed
-    const uint32_t bar_kempty = bar0 + 40;       // [KV_STAGES] QK^T that read the stage is done
-    const uint32_t bar_vempty = bar0 + 56;       // [KV_STAGES] PV that read the stage is done
-    const uint32_t bar_sfull = bar0 + 72;        // [2] scores ready in TMEM
-    const uint32_t bar_sempty = bar0 + 88;       // [2] softmax has read the scores (8 warps)
-    const uint32_t bar_pfull = bar0 + 104;       // [2] P written, O rescaled (8 warps)
-    const uint32_t bar_pempty = bar0 + 120;      // [2] PV done: P buffer free, O updated
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 136);
-    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 140);
+    const uint32_t bar_vfull = bar0 + 40;        // [KV_STAGES] V tile landed
+    const uint32_t bar_kempty = bar0 + 72;       // [KV_STAGES] QK^T that read the stage is done
+    const uint32_t bar_vempty = bar0 + 104;      // [KV_STAGES] PV that read the stage is done
+    const uint32_t bar_sfull = bar0 + 136;       // [2] scores ready in TMEM
+    const uint32_t bar_pfull = bar0 + 152;       // [2] P written over the scores, O rescaled (8 warps)
+    const uint32_t bar_pempty = bar0 + 168;      // [2] PV done: O updated
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 184);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 188);
     float* lx = reinterpret_cast<float*>(smem + L::OFF_LX);
 
     if (tid == 0) {
@@ -140,7 +137,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_sfull + 8 * i, 1);
-            mbar_init(bar_sempty + 8 * i, 8);
             mbar_init(bar_pfull + 8 * i, 8);
             mbar_init(bar_pempty + 8 * i, 1);
         }
@@ -155,12 +151,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tmem_relinquish();
     }
     if (MODE == MODE_DECODE) {
-        // rows >= G of the Q tile are never loaded and P rows of idle warps never written: zero them
+        // rows >= G of the Q tile are never loaded: zero them (their scores and weights stay 0)
         const uint4 z = make_uint4(0, 0, 0, 0);
         for (uint32_t i = tid; i < L::TILE / 16; i += ATTN_THREADS)
             reinterpret_cast<uint4*>(smem + L::OFF_Q)[i] = z;
-        for (uint32_t i = tid; i < 4 * L::ATOM / 16; i += ATTN_THREADS)
-            reinterpret_cast<uint4*>(smem + L::OFF_P)[i] = z;
         fence_proxy_async_smem();
     }
     tc_fence_before();
@@ -174,22 +168,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         return (MODE == MODE_DECODE || chunk_of(it) == 0) ? COL_OA : COL_OB;
     };
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+    if (warp == 0 || warp == 2) {
+        // ------------------------------------------------------------ TMA producers
+        // warp 0 streams Q and the K tiles, warp 2 the V tiles: a K tile is requested as soon as
+        // the QK^T that used its stage has finished, without queueing behind a wait for PV.
         if (lane == 0) {
-            if (MODE == MODE_DECODE) {
-                mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
-                for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
-            } else {
-                mbar_expect_tx(bar_q, L::TILE);
-                for (int a = 0; a < NATOM; ++a)
-                    tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
+            const int kv = (warp == 2) ? 1 : 0;
+            if (kv == 0) {
+                if (MODE == MODE_DECODE) {
+                    mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
+                    for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
+                } else {
+                    mbar_expect_tx(bar_q, L::TILE);
+                    for (int a = 0; a < NATOM; ++a)
+                        tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
+                }
             }
+            const CUtensorMap* tm = kv ? &tmV : &tmK;
             for (int it = 0; it < n_tiles; ++it) {
                 const int j = tile_first + it;
                 const int st = it % KV_STAGES;
                 const uint32_t use = it / KV_STAGES;
-                const uint32_t dK = sK + st * L::TILE, dV = sV + st * L::TILE;
+                const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
+                const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
+                const uint32_t empty = (kv ? bar_vempty : bar_kempty) + 8 * st;
                 int phys[8];
                 if (MODE != MODE_TRAIN) {
                     const int lp0 = (128 * j) / p.page_size;
@@ -206,22 +208,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         phys[i] = ph;
                     }
                 }
-                for (int kv = 0; kv < 2; ++kv) {
-                    const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
-                    const uint32_t empty = (kv ? bar_vempty : bar_kempty) + 8 * st;
-                    const uint32_t dst = kv ? dV : dK;
-                    const CUtensorMap* tm = kv ? &tmV : &tmK;
-                    if (use > 0) mbar_wait(empty, (use - 1) & 1, abort_word, p.dev_status);
-                    mbar_expect_tx(full, L::TILE);
-                    if (MODE == MODE_TRAIN) {
-                        const int row = static_cast<int>(tok0) + 128 * j;
-                        for (int a = 0; a < NATOM; ++a) tma_load_3d(dst + a * L::ATOM, tm, full, a * 64, kvh, row);
-                    } else {
-                        for (int i = 0; i < p.pages_per_tile; ++i) {
-                            const uint32_t off = static_cast<uint32_t>(i * p.page_size) * 128u;
-                            for (int a = 0; a < NATOM; ++a)
-                                tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, phys[i]);
-                        }
+                if (use > 0) mbar_wait(empty, (use - 1) & 1, abort_word, p.dev_status);
+                mbar_expect_tx(full, L::TILE);
+                if (MODE == MODE_TRAIN) {
+                    const int row = static_cast<int>(tok0) + 128 * j;
+                    for (int a = 0; a < NATOM; ++a) tma_load_3d(dst + a * L::ATOM, tm, full, a * 64, kvh, row);
+                } else {
+                    for (int i = 0; i < p.pages_per_tile; ++i) {
+                        const uint32_t off = static_cast<uint32_t>(i * p.page_size) * 128u;
+                        for (int a = 0; a < NATOM; ++a)
+                            tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, phys[i]);
                     }
                 }
             }
@@ -232,8 +228,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         if (lane == 0) {
             auto issue_qk = [&](int x) {
                 const int st = x % KV_STAGES, b = x & 1;
+                // S[b] still holds the weights of tile x-2; the PV that reads them was issued
+                // earlier by this thread, and MMAs of one thread execute in issue order
                 mbar_wait(bar_kfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
-                if (x >= 2) mbar_wait(bar_sempty + 8 * b, ((x >> 1) - 1) & 1, abort_word, p.dev_status);
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
@@ -253,8 +250,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const bool fresh = is_chunk_start(x);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t poff = b * 2 * L::ATOM + (ks >> 2) * L::ATOM + (ks & 3) * 32;
-                    mma_ss(tmem + col_o, smem_desc_sw128(sP + poff, 0, 1024),
+                    // A = bf16 weights in TMEM over the scores: 8 columns per 16 keys
+                    mma_ts(tmem + col_o, tmem + COL_S + 128 * b + 8 * ks,
                            smem_desc_sw128(sV + st * L::TILE + ks * 2048, L::ATOM, 1024), IDESC_PV,
                            (fresh && ks == 0) ? 0u : 1u);
                 }
@@ -333,36 +330,48 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const int kmax = qpos - 128 * j;            // columns > kmax are masked
                 const uint32_t ts = tlane + COL_S + 128 * b;
                 uint32_t own[64];
-                float mt = -CUDART_INF_F;
-                {   // the other half only contributes to the row maximum
-                    uint32_t oth[32];
+                uint32_t oth[32];
+                // own half (kept), first 32 columns of the other half (only for the row maximum)
+                tmem_ld32(ts + 64 * wg, *reinterpret_cast<uint32_t(*)[32]>(&own[0]));
+                tmem_ld32(ts + 64 * wg + 32, *reinterpret_cast<uint32_t(*)[32]>(&own[32]));
+                tmem_ld32(ts + 64 * (wg ^ 1), oth);
+                tmem_wait_ld();
+                float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+                const bool masked_tile = kmax < 127;
+                auto max_other = [&](int col0) {
+                    if (masked_tile) {
 #pragma unroll
-                    for (int cc = 0; cc < 2; ++cc) {
-                        tmem_ld32(ts + 64 * (wg ^ 1) + 32 * cc, oth);
-                        if (cc == 0) {
-                            tmem_ld32(ts + 64 * wg, *reinterpret_cast<uint32_t(*)[32]>(&own[0]));
-                            tmem_ld32(ts + 64 * wg + 32, *reinterpret_cast<uint32_t(*)[32]>(&own[32]));
-                        }
-                        tmem_wait_ld();
-                        const int col0 = 64 * (wg ^ 1) + 32 * cc;
-                        if (kmax >= 127) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) mt = fmaxf(mt, __uint_as_float(oth[i]));
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                mt = fmaxf(mt, (col0 + i > kmax) ? -CUDART_INF_F : __uint_as_float(oth[i]));
-                        }
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + i > kmax) oth[i] = 0xff800000u;      // -inf
                     }
-                }
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mx[k] = fmax3(mx[k], __uint_as_float(oth[i + 2 * k]), __uint_as_float(oth[i + 2 * k + 1]));
+                    }
+                };
+                max_other(64 * (wg ^ 1));
+                // second 32 columns of the other half arrive while the own half is reduced
+                tmem_ld32(ts + 64 * (wg ^ 1) + 32, oth);
                 const int own0 = 64 * wg;
-                if (kmax < 127) {
+                if (masked_tile) {
 #pragma unroll
                     for (int i = 0; i < 64; ++i)
                         if (own0 + i > kmax) own[i] = 0xff800000u;      // -inf
                 }
 #pragma unroll
-                for (int i = 0; i < 64; ++i) mt = fmaxf(mt, __uint_as_float(own[i]));
+                for (int i = 0; i < 64; i += 8) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mx[k] = fmax3(mx[k], __uint_as_float(own[i + 2 * k]), __uint_as_float(own[i + 2 * k + 1]));
+                }
+                tmem_wait_ld();
+                // rendezvous of the two threads of a row: once both have read all the scores they
+                // need, either may overwrite score columns with its weights
+                named_bar_sync(2 + quarter, 64);
+                max_other(64 * (wg ^ 1) + 32);
+                const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                 const float m_new = fmaxf(m_run, mt);
                 const float neg_mc = -__fmul_rn(m_new, c);
                 alpha = softmax_alpha(m_run, m_new, c);
@@ -380,20 +389,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 l_run = __fmaf_rn(l_run, alpha, rs.total());
                 m_run = m_new;
             }
-            // scores of this tile are in registers: release the TMEM buffer
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_sempty + 8 * b);
-            // the P buffer was last read by the PV of tile it-2
-            if (it >= 2) wait_pv(it - 2);
             if (active) {
-#pragma unroll
-                for (int q4 = 0; q4 < 8; ++q4) {
-                    const uint32_t off = L::OFF_P + (b * 2 + wg) * L::ATOM + r * 128 + ((q4 ^ (r & 7)) << 4);
-                    *reinterpret_cast<uint4*>(smem + off) =
-                        make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
-                }
-                fence_proxy_async_smem();
+                // weights go to TMEM over score columns that nobody reads any more
+                tmem_st32(tlane + COL_S + 128 * b + 32 * wg, pk);
             }
             if (fold_pending) {                       // uniform over the CTA
                 wait_pv(it - 1);
@@ -415,6 +413,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
                 tmem_wait_st();
             }
+            if (active) tmem_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pfull + 8 * b);

@@ -81,6 +81,13 @@ __device__ __forceinline__ void rowsum_add(RowSum8& s, int col, float p) {
     rowsum_add(s.h[col >> 6], col & 63, p);
 }
 
+// max of three (the maximum is exact, so its evaluation order is free)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
 // exponent argument of one score: s * c - mc, one fused multiply-add.
 __device__ __forceinline__ float softmax_p(float s, float c, float neg_mc) {
     return ex2_ftz(__fmaf_rn(s, c, neg_mc));
