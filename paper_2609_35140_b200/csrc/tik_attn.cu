@@ -6,7 +6,7 @@
 // order.  S = Q K^T and O += P V run on tcgen05 (M128 x N128 x K16 and M128 x Nd x K16,
 // fp32 accumulators in TMEM); Q, K, V arrive by TMA into 128B-swizzled shared memory
 // (K/V of the paged regimes are gathered page by page through the block table).  The CTA
-// is warp-specialised: one TMA warp, one MMA warp and two softmax warpgroups that each own
+// is warp-specialised: two TMA warps (K, V), two MMA warps (QK^T, PV) and two softmax warpgroups that each own
 // 64 of a tile's 128 key columns (and half of the O columns), working straight out of TMEM
 // with the arithmetic of tik_core.cuh; scores are double-buffered so the QK^T of tile j+1
 // runs under the softmax of tile j.  What differs between regimes is only where rows come from and where they
@@ -25,7 +25,7 @@ namespace tik {
 
 enum { MODE_TRAIN = 0, MODE_PREFILL = 1, MODE_DECODE = 2 };
 
-constexpr int ATTN_THREADS = 384;   // warp 0 TMA (Q, K), warp 1 MMA, warp 2 TMA (V), warp 3 idle, warps 4-11 softmax
+constexpr int ATTN_THREADS = 384;   // warp 0 TMA (Q, K), warp 1 QK^T MMA, warp 2 TMA (V), warp 3 PV MMA, warps 4-11 softmax
 constexpr int KV_STAGES = 3;
 
 template <int D>
@@ -120,9 +120,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const uint32_t bar_vfull = bar0 + 40;        // [KV_STAGES] V tile landed
     const uint32_t bar_kempty = bar0 + 72;       // [KV_STAGES] QK^T that read the stage is done
     const uint32_t bar_vempty = bar0 + 104;      // [KV_STAGES] PV that read the stage is done
-    const uint32_t bar_sfull = bar0 + 136;       // [2] scores ready in TMEM
+    const uint32_t bar_sfull = bar0 + 136;       // [2] QK^T done: scores ready in TMEM
     const uint32_t bar_pfull = bar0 + 152;       // [2] P written over the scores, O rescaled (8 warps)
-    const uint32_t bar_pempty = bar0 + 168;      // [2] PV done: O updated
+    const uint32_t bar_pempty = bar0 + 168;      // [2] PV done: O updated, score buffer free
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 184);
     volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 188);
     float* lx = reinterpret_cast<float*>(smem + L::OFF_LX);
@@ -191,7 +191,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const uint32_t use = it / KV_STAGES;
                 const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
                 const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
-                const uint32_t empty = (kv ? bar_vempty : bar_kempty) + 8 * st;
                 int phys[8];
                 if (MODE != MODE_TRAIN) {
                     const int lp0 = (128 * j) / p.page_size;
@@ -208,7 +207,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         phys[i] = ph;
                     }
                 }
-                if (use > 0) mbar_wait(empty, (use - 1) & 1, abort_word, p.dev_status);
+                // Each stage has its own release barrier with this thread as its only waiter: a
+                // barrier shared with waiters of a different lag could run two phases ahead of
+                // the slowest one, which a parity wait cannot tell from "not yet".
+                if (use > 0)
+                    mbar_wait((kv ? bar_vempty : bar_kempty) + 8 * st, (use - 1) & 1, abort_word, p.dev_status);
                 mbar_expect_tx(full, L::TILE);
                 if (MODE == MODE_TRAIN) {
                     const int row = static_cast<int>(tok0) + 128 * j;
@@ -224,45 +227,41 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ QK^T issuer
+        // Two threads feed the tensor pipe (this one and the PV issuer in warp 3): whatever an
+        // issuing thread executes between MMAs is time in which it queues nothing, so each
+        // keeps to waits, one MMA chain and one commit per tile.
         if (lane == 0) {
-            auto issue_qk = [&](int x) {
+            mbar_wait(bar_q, 0, abort_word, p.dev_status);
+            const uint64_t dq = smem_desc_sw128(sQ, 0, 1024);
+            for (int x = 0; x < n_tiles; ++x) {
                 const int st = x % KV_STAGES, b = x & 1;
-                // S[b] still holds the weights of tile x-2; the PV that reads them was issued
-                // earlier by this thread, and MMAs of one thread execute in issue order
+                // S[b] holds the weights of tile x-2 until its PV has completed
+                if (x >= 2) mbar_wait(bar_pempty + 8 * b, ((x >> 1) - 1) & 1, abort_word, p.dev_status);
                 mbar_wait(bar_kfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
                 tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t koff = (ks >> 2) * L::ATOM + (ks & 3) * 32;
-                    mma_ss(tmem + COL_S + 128 * b, smem_desc_sw128(sQ + koff, 0, 1024),
-                           smem_desc_sw128(sK + st * L::TILE + koff, 0, 1024), IDESC_QK, ks > 0);
-                }
+                const uint64_t dk = smem_desc_sw128(sK + st * L::TILE, 0, 1024);
+                if (D == 128) mma_ss_chain8_fresh(tmem + COL_S + 128 * b, dq, dk, IDESC_QK);
+                else mma_ss_chain4_fresh(tmem + COL_S + 128 * b, dq, dk, IDESC_QK);
                 mma_commit(bar_sfull + 8 * b);
                 mma_commit(bar_kempty + 8 * st);
-            };
-            auto issue_pv = [&](int x) {
+            }
+        }
+        __syncwarp();
+    } else if (warp == 3) {
+        // ------------------------------------------------------------ PV issuer
+        if (lane == 0) {
+            for (int x = 0; x < n_tiles; ++x) {
                 const int st = x % KV_STAGES, b = x & 1;
                 mbar_wait(bar_vfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
                 mbar_wait(bar_pfull + 8 * b, (x >> 1) & 1, abort_word, p.dev_status);
                 tc_fence_after();
-                const uint32_t col_o = col_o_of(x);
-                const bool fresh = is_chunk_start(x);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    // A = bf16 weights in TMEM over the scores: 8 columns per 16 keys
-                    mma_ts(tmem + col_o, tmem + COL_S + 128 * b + 8 * ks,
-                           smem_desc_sw128(sV + st * L::TILE + ks * 2048, L::ATOM, 1024), IDESC_PV,
-                           (fresh && ks == 0) ? 0u : 1u);
-                }
-                mma_commit(bar_vempty + 8 * st);
+                // A = bf16 weights in TMEM over the scores (8 columns per 16 keys), B = V tile
+                mma_ts_chain8(tmem + col_o_of(x), tmem + COL_S + 128 * b,
+                              smem_desc_sw128(sV + st * L::TILE, L::ATOM, 1024), IDESC_PV,
+                              is_chunk_start(x) ? 0u : 1u);
                 mma_commit(bar_pempty + 8 * b);
-            };
-            mbar_wait(bar_q, 0, abort_word, p.dev_status);
-            issue_qk(0);
-            for (int it = 0; it < n_tiles; ++it) {
-                if (it + 1 < n_tiles) issue_qk(it + 1);
-                issue_pv(it);
+                mma_commit(bar_vempty + 8 * st);
             }
         }
         __syncwarp();

@@ -117,10 +117,8 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     mbar_wait(bar_full + 8 * s, (it / STAGES) & 1, abort_word, p.dev_status);
                     tc_fence_after();
                     const uint32_t a0 = sbase + s * STAGE_BYTES, b0 = a0 + A_BYTES;
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma_ss(tmem + buf * 128, smem_desc_sw128(a0 + ks * 32, 0, 1024),
-                               smem_desc_sw128(b0 + ks * 32, 0, 1024), IDESC, (kb | ks) ? 1u : 0u);
+                    mma_ss_chain4(tmem + buf * 128, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
+                                  IDESC, kb ? 1u : 0u);
                     mma_commit(bar_empty + 8 * s);
                 }
                 mma_commit(bar_acc_full + 8 * buf);

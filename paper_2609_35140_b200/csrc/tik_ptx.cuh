@@ -206,6 +206,63 @@ __device__ __forceinline__ void named_bar_arrive(uint32_t id, uint32_t nthreads)
 __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
+// ---- MMA chains issued from one asm block.  The issuing thread's own instruction stream
+// limits how fast MMAs enter the tensor pipe, so a chain spends two 64-bit adds per MMA on
+// descriptor stepping and nothing else.  Offsets are in descriptor units (16 bytes).
+#define TIK_MMA_SS_STEP(OFFA, OFFB)                                   \
+    "add.u64 da, %1, " #OFFA ";\n\t"                                  \
+    "add.u64 db, %2, " #OFFB ";\n\t"                                  \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, pt;\n\t"
+
+// K-major A and B, 64-wide K slice inside one 128B-swizzle atom: 4 steps of 32 bytes.
+// first_accumulate == 0 makes the first MMA overwrite D.
+__device__ __forceinline__ void mma_ss_chain4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                              uint32_t idesc, uint32_t first_accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p0, pt;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p0, %4, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p0;\n\t"
+        TIK_MMA_SS_STEP(2, 2) TIK_MMA_SS_STEP(4, 4) TIK_MMA_SS_STEP(6, 6)
+        "}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(first_accumulate)
+        : "memory");
+}
+// Same for a 128-wide K (two atoms 16 KiB = 1024 units apart): 8 steps, first one overwrites D.
+__device__ __forceinline__ void mma_ss_chain8_fresh(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                    uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p0, pt;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p0;\n\t"
+        TIK_MMA_SS_STEP(2, 2) TIK_MMA_SS_STEP(4, 4) TIK_MMA_SS_STEP(6, 6)
+        TIK_MMA_SS_STEP(1024, 1024) TIK_MMA_SS_STEP(1026, 1026) TIK_MMA_SS_STEP(1028, 1028)
+        TIK_MMA_SS_STEP(1030, 1030)
+        "}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ss_chain4_fresh(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                    uint32_t idesc) {
+    mma_ss_chain4(d_tmem, a_desc, b_desc, idesc, 0u);
+}
+
+// A from TMEM (8 columns per step), B = MN-major tile whose 16-key steps are 2 KiB = 128 units
+// apart: the 8 steps of one 128-key tile.  first_accumulate == 0 overwrites D on the first step.
+#define TIK_MMA_TS_STEP(OFFA, OFFB)                                   \
+    "add.u32 ta, %1, " #OFFA ";\n\t"                                  \
+    "add.u64 db, %2, " #OFFB ";\n\t"                                  \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, pt;\n\t"
+__device__ __forceinline__ void mma_ts_chain8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                              uint32_t idesc, uint32_t first_accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p0, pt;\n\t.reg .b64 db;\n\t.reg .b32 ta;\n\t"
+        "setp.ne.b32 p0, %4, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+        TIK_MMA_TS_STEP(8, 128) TIK_MMA_TS_STEP(16, 256) TIK_MMA_TS_STEP(24, 384)
+        TIK_MMA_TS_STEP(32, 512) TIK_MMA_TS_STEP(40, 640) TIK_MMA_TS_STEP(48, 768)
+        TIK_MMA_TS_STEP(56, 896)
+        "}" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(first_accumulate)
+        : "memory");
+}
+
 // Arrives on the mbarrier once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
