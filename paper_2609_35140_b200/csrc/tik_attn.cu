@@ -6,11 +6,12 @@
 // order.  S = Q K^T and O += P V run on tcgen05 (M128 x N128 x K16 and M128 x Nd x K16,
 // fp32 accumulators in TMEM); Q, K, V arrive by TMA into 128B-swizzled shared memory
 // (K/V of the paged regimes are gathered page by page through the block table).  The CTA
-// is warp-specialised: two TMA warps (K, V), two MMA warps (QK^T, PV) and two softmax warpgroups that each own
-// 64 of a tile's 128 key columns (and half of the O columns), working straight out of TMEM
-// with the arithmetic of tik_core.cuh; scores are double-buffered so the QK^T of tile j+1
-// runs under the softmax of tile j.  What differs between regimes is only where rows come from and where they
-// go:
+// is warp-specialised: two TMA warps (K, V), two MMA-issuing warps (QK^T, PV) and two
+// softmax warpgroups that alternate over KV tiles, one thread per row, working straight out
+// of TMEM with the arithmetic of tik_core.cuh.  A thread pulls its score row into registers
+// and releases the score buffer at once, and the bf16 weights go to two TMEM buffers of their
+// own, so the QK^T of tile j+1 and the PV of tile j-1 run under the softmax of tile j.  What differs between regimes is only where rows come from
+// and where they go:
 //   train   : rows = 128 consecutive tokens of one (sequence, query head); K/V packed
 //   prefill : same rows, aligned to absolute positions; K/V from pages
 //   decode  : rows 0..G-1 = the G query heads of one KV head for one sequence (other rows
@@ -36,9 +37,9 @@ struct AttnSmem {
     static constexpr uint32_t OFF_K = TILE;
     static constexpr uint32_t OFF_V = OFF_K + KV_STAGES * TILE;
     static constexpr uint32_t OFF_BAR = OFF_V + KV_STAGES * TILE;
-    static constexpr uint32_t OFF_LX = OFF_BAR + 256;             // 2 x 128 floats: half row sums
-    static constexpr uint32_t BYTES = OFF_LX + 1024;
-    static constexpr uint32_t ALLOC = BYTES + 1024;               // slack for 1 KiB alignment
+    static constexpr uint32_t OFF_LX = OFF_BAR + 272;             // 3 x 128 floats of row state
+    static constexpr uint32_t BYTES = OFF_LX + 3 * 512;
+    static constexpr uint32_t ALLOC = BYTES;                      // base must be 1 KiB aligned
 };
 
 template <int D, int MODE>
@@ -49,7 +50,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     constexpr int NATOM = D / 64;
     constexpr int DH = D / 2;                              // O columns owned by one softmax thread
     constexpr uint32_t TMEM_COLS = 512;
-    constexpr uint32_t COL_S = 0;                          // two score buffers of 128 columns
+    constexpr uint32_t COL_S = 0;                          // one score buffer of 128 columns
+    constexpr uint32_t COL_P = 128;                        // two weight buffers of 64 columns (bf16 pairs)
     constexpr uint32_t COL_OA = 256, COL_OB = 256 + D;
     constexpr uint32_t IDESC_QK = mma_idesc_bf16(128, 128, false);
     constexpr uint32_t IDESC_PV = mma_idesc_bf16(128, D, true);
@@ -107,11 +109,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const int n_tiles = tile_last - tile_first + 1;
 
     // ---------------------------------------------------------------- shared memory
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw_addr = smem_u32(smem_raw);
-    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
-    uint8_t* smem = smem_raw + pad;
-    const uint32_t sbase = raw_addr + pad;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = smem_raw;
+    const uint32_t sbase = smem_u32(smem_raw);
+    if (sbase & 1023u) {     // the swizzled tiles need a 1 KiB aligned base: refuse to run otherwise
+        if (tid == 0) atomicOr(p.dev_status, TIK_DEV_WAIT_EXPIRED);
+        return;
+    }
     const uint32_t sQ = sbase + L::OFF_Q, sK = sbase + L::OFF_K, sV = sbase + L::OFF_V;
     // barriers (8 bytes each)
     const uint32_t bar0 = sbase + L::OFF_BAR;
@@ -120,11 +124,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const uint32_t bar_vfull = bar0 + 40;        // [KV_STAGES] V tile landed
     const uint32_t bar_kempty = bar0 + 72;       // [KV_STAGES] QK^T that read the stage is done
     const uint32_t bar_vempty = bar0 + 104;      // [KV_STAGES] PV that read the stage is done
-    const uint32_t bar_sfull = bar0 + 136;       // [2] QK^T done: scores ready in TMEM
-    const uint32_t bar_pfull = bar0 + 152;       // [2] P written over the scores, O rescaled (8 warps)
-    const uint32_t bar_pempty = bar0 + 168;      // [2] PV done: O updated, score buffer free
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 184);
-    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 188);
+    const uint32_t bar_sfull = bar0 + 136;       // [2] QK^T of an even / odd tile done: scores ready in TMEM
+    const uint32_t bar_pfull = bar0 + 152;       // [2] P written over the scores, O rescaled (4 warps)
+    const uint32_t bar_pempty = bar0 + 168;      // [2] PV done: O updated, weight buffer free
+    const uint32_t bar_hand = bar0 + 184;        // [2][4] row-state hand-off between the warpgroups
+    const uint32_t bar_sempty = bar0 + 248;      // [2] scores of a tile are in registers (4 warps)
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 264);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 268);
     float* lx = reinterpret_cast<float*>(smem + L::OFF_LX);
 
     if (tid == 0) {
@@ -137,9 +143,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_sfull + 8 * i, 1);
-            mbar_init(bar_pfull + 8 * i, 8);
+            mbar_init(bar_pfull + 8 * i, 4);
+            mbar_init(bar_sempty + 8 * i, 4);
             mbar_init(bar_pempty + 8 * i, 1);
         }
+        for (int i = 0; i < 8; ++i) mbar_init(bar_hand + 8 * i, 1);
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmQ);
@@ -236,13 +244,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             const uint64_t dq = smem_desc_sw128(sQ, 0, 1024);
             for (int x = 0; x < n_tiles; ++x) {
                 const int st = x % KV_STAGES, b = x & 1;
-                // S[b] holds the weights of tile x-2 until its PV has completed
-                if (x >= 2) mbar_wait(bar_pempty + 8 * b, ((x >> 1) - 1) & 1, abort_word, p.dev_status);
+                // the single score buffer is free once the softmax of tile x-1 holds it in registers
+                if (x >= 1) mbar_wait(bar_sempty + 8 * ((x - 1) & 1), ((x - 1) >> 1) & 1, abort_word, p.dev_status);
                 mbar_wait(bar_kfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
                 tc_fence_after();
                 const uint64_t dk = smem_desc_sw128(sK + st * L::TILE, 0, 1024);
-                if (D == 128) mma_ss_chain8_fresh(tmem + COL_S + 128 * b, dq, dk, IDESC_QK);
-                else mma_ss_chain4_fresh(tmem + COL_S + 128 * b, dq, dk, IDESC_QK);
+                if (D == 128) mma_ss_chain8_fresh(tmem + COL_S, dq, dk, IDESC_QK);
+                else mma_ss_chain4_fresh(tmem + COL_S, dq, dk, IDESC_QK);
                 mma_commit(bar_sfull + 8 * b);
                 mma_commit(bar_kempty + 8 * st);
             }
@@ -256,8 +264,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 mbar_wait(bar_vfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
                 mbar_wait(bar_pfull + 8 * b, (x >> 1) & 1, abort_word, p.dev_status);
                 tc_fence_after();
-                // A = bf16 weights in TMEM over the scores (8 columns per 16 keys), B = V tile
-                mma_ts_chain8(tmem + col_o_of(x), tmem + COL_S + 128 * b,
+                // A = bf16 weights in TMEM (8 columns per 16 keys), B = V tile
+                mma_ts_chain8(tmem + col_o_of(x), tmem + COL_P + 64 * b,
                               smem_desc_sw128(sV + st * L::TILE, L::ATOM, 1024), IDESC_PV,
                               is_chunk_start(x) ? 0u : 1u);
                 mma_commit(bar_pempty + 8 * b);
@@ -267,170 +275,214 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         __syncwarp();
     } else if (warp >= 4) {
         // ------------------------------------------------------------ softmax (two warpgroups)
-        const int wg = (warp - 4) >> 2;                     // owns key columns [64 wg, 64 wg + 64)
+        // The warpgroups alternate over KV tiles: warpgroup wg owns the tiles with it % 2 == wg
+        // and with them score buffer wg, one thread per row and all 128 columns of the tile.
+        // While one warpgroup is in its exp2 phase the other loads scores, reduces the maximum
+        // and stores weights, so the special-function unit stays busy.  The row state (running
+        // maximum, the two half row sums, the folded state of earlier chunks) lives in shared
+        // memory and is handed from the thread of tile it to the thread of tile it+1 through
+        // two mbarriers per lane quarter.
+        const int wg = (warp - 4) >> 2;
         const int quarter = warp & 3;                       // TMEM lane quarter of this warp
         const int r = quarter * 32 + lane;                  // tile row == TMEM lane
         const uint32_t tlane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const int qpos = (MODE == MODE_DECODE) ? (ctx - 1) : (128 * T + r);
         const bool active = (MODE != MODE_DECODE) || (quarter == 0);
         const float c = p.c;
-        float m_run = -CUDART_INF_F, l_run = 0.0f;          // current chunk (l: this thread's half)
-        float m_prev = 0.0f, l_prev = 0.0f;                  // finished chunk waiting to be folded
-        float M_g = -CUDART_INF_F, L_g = 0.0f;               // folded state of earlier chunks
-        bool fold_pending = false;
-        int prev_chunk = 0;
+        float* st_m = lx;                 // [128]    running maximum of the current chunk
+        float* st_l = lx + 128;           // [2][128] half row sums of the current chunk
+        const uint32_t bar_m = bar_hand + 8 * quarter;       // "maximum of tile it published"
+        const uint32_t bar_l = bar_hand + 32 + 8 * quarter;  // "row sums of tile it published"
+        const uint32_t ts = tlane + COL_S;
+        const uint32_t tp = tlane + COL_P + 64 * wg;
+        // Folded state of the finished chunks.  Both threads of a row keep it: warpgroup 0 folds
+        // at the first tile of a chunk (the state of the finished chunk is handed to it), and
+        // warpgroup 1 owns every chunk's last tile, so it folds the same numbers on its own.
+        float M_g = -CUDART_INF_F, Lg_lo = 0.0f, Lg_hi = 0.0f;
+        float m_own = -CUDART_INF_F, l_own_lo = 0.0f, l_own_hi = 0.0f;   // state after this thread's last tile
 
-        // waits until the PV of tile `x` has completed (O and the P buffer are consistent)
         auto wait_pv = [&](int x) {
             mbar_wait(bar_pempty + 8 * (x & 1), (x >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
         };
-        // folds the finished chunk (m_prev, l_prev, O_B) into the global state; PV must be done
-        auto fold_chunk = [&]() {
-            if (prev_chunk == 0) {           // chunk 0 accumulated in place in O_A
-                M_g = m_prev;
-                L_g = l_prev;
+        // folds a finished chunk (m_c, l_c halves) into the global row state; with_o also folds
+        // its accumulator O_B into O_A (one thread per row does that, after the chunk's last PV)
+        auto fold_chunk = [&](int chunk_idx, float m_c, float l_c_lo, float l_c_hi, bool with_o) {
+            if (chunk_idx == 0) {            // chunk 0 accumulated in place in O_A
+                M_g = m_c;
+                Lg_lo = l_c_lo;
+                Lg_hi = l_c_hi;
             } else {
-                const FoldCoef f = fold_coef(M_g, m_prev, c);
-                L_g = fold_value(L_g, l_prev, f);
+                const FoldCoef f = fold_coef(M_g, m_c, c);
+                Lg_lo = fold_value(Lg_lo, l_c_lo, f);
+                Lg_hi = fold_value(Lg_hi, l_c_hi, f);
                 M_g = f.M_new;
+                if (with_o) {
 #pragma unroll
-                for (int cc = 0; cc < DH / 32; ++cc) {
-                    uint32_t a[32], b[32];
-                    tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, a);
-                    tmem_ld32(tlane + COL_OB + DH * wg + 32 * cc, b);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        a[i] = __float_as_uint(fold_value(__uint_as_float(a[i]), __uint_as_float(b[i]), f));
-                    tmem_st32(tlane + COL_OA + DH * wg + 32 * cc, a);
-                }
-                tmem_wait_st();
-            }
-        };
-
-        for (int it = 0; it < n_tiles; ++it) {
-            const int j = tile_first + it;
-            const int b = it & 1;
-            const bool chunk_start = is_chunk_start(it);
-            if (MODE != MODE_DECODE && chunk_start && it > 0) {
-                m_prev = m_run;
-                l_prev = l_run;
-                prev_chunk = chunk_of(it - 1);
-                fold_pending = true;
-                m_run = -CUDART_INF_F;
-                l_run = 0.0f;
-            }
-            mbar_wait(bar_sfull + 8 * b, (it >> 1) & 1, abort_word, p.dev_status);
-            tc_fence_after();
-            uint32_t pk[32];
-            float alpha = 1.0f;
-            if (active) {
-                const int kmax = qpos - 128 * j;            // columns > kmax are masked
-                const uint32_t ts = tlane + COL_S + 128 * b;
-                uint32_t own[64];
-                uint32_t oth[32];
-                // own half (kept), first 32 columns of the other half (only for the row maximum)
-                tmem_ld32(ts + 64 * wg, *reinterpret_cast<uint32_t(*)[32]>(&own[0]));
-                tmem_ld32(ts + 64 * wg + 32, *reinterpret_cast<uint32_t(*)[32]>(&own[32]));
-                tmem_ld32(ts + 64 * (wg ^ 1), oth);
-                tmem_wait_ld();
-                float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-                const bool masked_tile = kmax < 127;
-                auto max_other = [&](int col0) {
-                    if (masked_tile) {
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        uint32_t a[32], b[32];
+                        tmem_ld32(tlane + COL_OA + 32 * cc, a);
+                        tmem_ld32(tlane + COL_OB + 32 * cc, b);
+                        tmem_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
-                            if (col0 + i > kmax) oth[i] = 0xff800000u;      // -inf
+                            a[i] = __float_as_uint(fold_value(__uint_as_float(a[i]), __uint_as_float(b[i]), f));
+                        tmem_st32(tlane + COL_OA + 32 * cc, a);
                     }
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            mx[k] = fmax3(mx[k], __uint_as_float(oth[i + 2 * k]), __uint_as_float(oth[i + 2 * k + 1]));
-                    }
-                };
-                max_other(64 * (wg ^ 1));
-                // second 32 columns of the other half arrive while the own half is reduced
-                tmem_ld32(ts + 64 * (wg ^ 1) + 32, oth);
-                const int own0 = 64 * wg;
-                if (masked_tile) {
-#pragma unroll
-                    for (int i = 0; i < 64; ++i)
-                        if (own0 + i > kmax) own[i] = 0xff800000u;      // -inf
+                    tmem_wait_st();
                 }
+            }
+        };
+        const int last = n_tiles - 1;
+
+        for (int it = wg; it < n_tiles; it += 2) {
+            const int j = tile_first + it;
+            const bool chunk_start = is_chunk_start(it);
+            mbar_wait(bar_sfull + 8 * wg, (it >> 1) & 1, abort_word, p.dev_status);
+            // The weight buffer of this warpgroup was last read by the PV of tile it-2.  Every
+            // warp waits for it, idle ones too: it also keeps a warp from arriving for tile it on
+            // a barrier whose phase for tile it-2 is still collecting arrivals.
+            if (it >= 2) wait_pv(it - 2);
+            tc_fence_after();
+            if (active) {
+                const int kmax = qpos - 128 * j;            // columns > kmax are masked
+                uint32_t sc[128];
+                tmem_ld32(ts, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+                tmem_ld32(ts + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[32]));
+                tmem_ld32(ts + 64, *reinterpret_cast<uint32_t(*)[32]>(&sc[64]));
+                tmem_ld32(ts + 96, *reinterpret_cast<uint32_t(*)[32]>(&sc[96]));
+                tmem_wait_ld();
+                // the scores are in registers: the next QK^T may overwrite the buffer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_sempty + 8 * wg);
+                if (kmax < 127) {
 #pragma unroll
-                for (int i = 0; i < 64; i += 8) {
+                    for (int i = 0; i < 128; ++i)
+                        if (i > kmax) sc[i] = 0xff800000u;          // -inf
+                }
+                float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+                for (int i = 0; i < 128; i += 8) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        mx[k] = fmax3(mx[k], __uint_as_float(own[i + 2 * k]), __uint_as_float(own[i + 2 * k + 1]));
+                        mx[k] = fmax3(mx[k], __uint_as_float(sc[i + 2 * k]), __uint_as_float(sc[i + 2 * k + 1]));
                 }
-                tmem_wait_ld();
-                // rendezvous of the two threads of a row: once both have read all the scores they
-                // need, either may overwrite score columns with its weights
-                named_bar_sync(2 + quarter, 64);
-                max_other(64 * (wg ^ 1) + 32);
                 const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                const float m_new = fmaxf(m_run, mt);
+                // state handed over by the thread that processed tile it-1
+                float m_old = -CUDART_INF_F, l_old_lo = 0.0f, l_old_hi = 0.0f;
+                float m_prev = 0.0f, l_prev_lo = 0.0f, l_prev_hi = 0.0f;   // finished chunk, if any
+                const bool fold_now = (MODE != MODE_DECODE) && chunk_start && it > 0;
+                if (it > 0) {
+                    mbar_wait(bar_m, (it - 1) & 1, abort_word, p.dev_status);
+                    if (fold_now) {
+                        mbar_wait(bar_l, (it - 1) & 1, abort_word, p.dev_status);
+                        m_prev = st_m[r];
+                        l_prev_lo = st_l[r];
+                        l_prev_hi = st_l[128 + r];
+                    } else {
+                        m_old = st_m[r];
+                    }
+                }
+                const float m_new = fmaxf(m_old, mt);
+                st_m[r] = m_new;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_m);
                 const float neg_mc = -__fmul_rn(m_new, c);
-                alpha = softmax_alpha(m_run, m_new, c);
-                RowSum4 rs;
-                rs.reset();
+                const float alpha = softmax_alpha(m_old, m_new, c);
+                RowSum4 rs_lo, rs_hi;
+                rs_lo.reset();
+                rs_hi.reset();
 #pragma unroll
                 for (int i = 0; i < 64; i += 2) {
                     // a masked score is -inf: fma gives -inf and ex2 gives +0 exactly
-                    const float p0 = softmax_p(__uint_as_float(own[i]), c, neg_mc);
-                    const float p1 = softmax_p(__uint_as_float(own[i + 1]), c, neg_mc);
-                    rowsum_add(rs, i, p0);
-                    rowsum_add(rs, i + 1, p1);
-                    pk[i >> 1] = pack_bf16x2(p0, p1);
+                    const float p0 = softmax_p(__uint_as_float(sc[i]), c, neg_mc);
+                    const float p1 = softmax_p(__uint_as_float(sc[i + 1]), c, neg_mc);
+                    rowsum_add(rs_lo, i, p0);
+                    rowsum_add(rs_lo, i + 1, p1);
+                    sc[i >> 1] = pack_bf16x2(p0, p1);
                 }
-                l_run = __fmaf_rn(l_run, alpha, rs.total());
-                m_run = m_new;
-            }
-            if (active) {
-                // weights go to TMEM over score columns that nobody reads any more
-                tmem_st32(tlane + COL_S + 128 * b + 32 * wg, pk);
-            }
-            if (fold_pending) {                       // uniform over the CTA
-                wait_pv(it - 1);
-                if (active) fold_chunk();
-                fold_pending = false;
-            } else if (!chunk_start && active && !__all_sync(0xffffffffu, alpha == 1.0f)) {
-                // rescale this thread's half of the chunk accumulator
-                wait_pv(it - 1);
-                const uint32_t to = tlane + col_o_of(it) + DH * wg;
+                tmem_st32(tp, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
 #pragma unroll
-                for (int cc = 0; cc < DH / 32; ++cc) {
-                    uint32_t v[32];
-                    tmem_ld32(to + 32 * cc, v);
-                    tmem_wait_ld();
+                for (int i = 0; i < 64; i += 2) {
+                    const float p0 = softmax_p(__uint_as_float(sc[64 + i]), c, neg_mc);
+                    const float p1 = softmax_p(__uint_as_float(sc[64 + i + 1]), c, neg_mc);
+                    rowsum_add(rs_hi, i, p0);
+                    rowsum_add(rs_hi, i + 1, p1);
+                    sc[32 + (i >> 1)] = pack_bf16x2(p0, p1);
+                }
+                tmem_st32(tp + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[32]));
+                if (it > 0 && !fold_now) {
+                    mbar_wait(bar_l, (it - 1) & 1, abort_word, p.dev_status);
+                    if (!chunk_start) {
+                        l_old_lo = st_l[r];
+                        l_old_hi = st_l[128 + r];
+                    }
+                }
+                m_own = m_new;
+                l_own_lo = __fmaf_rn(l_old_lo, alpha, rs_lo.total());
+                l_own_hi = __fmaf_rn(l_old_hi, alpha, rs_hi.total());
+                st_l[r] = l_own_lo;
+                st_l[128 + r] = l_own_hi;
+                if (fold_now) {
+                    wait_pv(it - 1);
+                    fold_chunk(chunk_of(it - 1), m_prev, l_prev_lo, l_prev_hi, true);
+                } else if (!chunk_start && !__all_sync(0xffffffffu, alpha == 1.0f)) {
+                    // rescale the chunk accumulator of this row
+                    wait_pv(it - 1);
+                    const uint32_t to = tlane + col_o_of(it);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
-                    tmem_st32(to + 32 * cc, v);
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        uint32_t v[32];
+                        tmem_ld32(to + 32 * cc, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
+                        tmem_st32(to + 32 * cc, v);
+                    }
                 }
                 tmem_wait_st();
+                // this thread closed a chunk that is not the row's last: fold its scalars here too
+                if (MODE != MODE_DECODE && it != last && ((tile_first + it) % TILES_PER_CHUNK) == TILES_PER_CHUNK - 1)
+                    fold_chunk(chunk_of(it), m_own, l_own_lo, l_own_hi, false);
             }
-            if (active) tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_pfull + 8 * b);
+            if (lane == 0) {
+                if (!active) mbar_arrive(bar_sempty + 8 * wg);
+                mbar_arrive(bar_pfull + 8 * wg);
+                if (active) mbar_arrive(bar_l);
+            }
         }
 
-        // ---- all tiles issued: wait for the last PV, then finish the row
-        wait_pv(n_tiles - 1);
-        if (MODE == MODE_DECODE) {
-            if (active && r < p.G) {
-                const long long slot = (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk;
-                if (wg == 0) {
-                    p.part_ml[4 * slot] = m_run;
-                    p.part_ml[4 * slot + 1] = l_run;
+        // ---- the warpgroup that owned the last tile finishes the row state
+        if (wg == (last & 1)) {
+            wait_pv(last);
+            if (active) {
+                if (MODE == MODE_DECODE) {
+                    if (r < p.G) {
+                        const long long slot =
+                            (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk;
+                        p.part_ml[4 * slot] = m_own;
+                        p.part_ml[4 * slot + 1] = l_own_lo;
+                        p.part_ml[4 * slot + 2] = l_own_hi;
+                    }
                 } else {
-                    p.part_ml[4 * slot + 2] = l_run;
+                    fold_chunk(chunk_of(last), m_own, l_own_lo, l_own_hi, true);
+                    const float Ltot = finalize_l(Lg_lo, Lg_hi);
+                    st_m[r] = finalize_inv(Ltot);       // the hand-off slots are free now
+                    const bool valid = (r >= row_lo) && (r < row_hi);
+                    if (valid && p.lse) p.lse[(qrow0 + r) * p.Hq + head] = finalize_lse(M_g, Ltot, c);
                 }
             }
-            if (active) {
+            tc_fence_before();
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        tc_fence_after();
+        // both warpgroups write half of the output columns each
+        if (active) {
+            if (MODE == MODE_DECODE) {
 #pragma unroll
                 for (int cc = 0; cc < DH / 32; ++cc) {
                     uint32_t v[32];
@@ -446,39 +498,29 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                                                  __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
                     }
                 }
-            }
-        } else {
-            m_prev = m_run;
-            l_prev = l_run;
-            prev_chunk = chunk_of(n_tiles - 1);
-            fold_chunk();
-            // exchange the half row sums between the two threads of a row
-            lx[wg * 128 + r] = L_g;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            const float l_lo = lx[r], l_hi = lx[128 + r];
-            const float Ltot = finalize_l(l_lo, l_hi);
-            const float inv = finalize_inv(Ltot);
-            const bool valid = (r >= row_lo) && (r < row_hi);
-            const long long orow = (qrow0 + r) * p.Hq + head;
-            __nv_bfloat16* optr = reinterpret_cast<__nv_bfloat16*>(p.o) + orow * D + DH * wg;
+            } else {
+                const float inv = st_m[r];
+                const bool valid = (r >= row_lo) && (r < row_hi);
+                const long long orow = (qrow0 + r) * p.Hq + head;
+                __nv_bfloat16* optr = reinterpret_cast<__nv_bfloat16*>(p.o) + orow * D + DH * wg;
 #pragma unroll
-            for (int cc = 0; cc < DH / 32; ++cc) {
-                uint32_t v[32];
-                tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, v);
-                tmem_wait_ld();
-                if (valid) {
-                    uint32_t o16[16];
+                for (int cc = 0; cc < DH / 32; ++cc) {
+                    uint32_t v[32];
+                    tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, v);
+                    tmem_wait_ld();
+                    if (valid) {
+                        uint32_t o16[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        o16[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv),
-                                             finalize_o(__uint_as_float(v[2 * i + 1]), inv));
-                    uint4* dst = reinterpret_cast<uint4*>(optr + 32 * cc);
+                        for (int i = 0; i < 16; ++i)
+                            o16[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv),
+                                                 finalize_o(__uint_as_float(v[2 * i + 1]), inv));
+                        uint4* dst = reinterpret_cast<uint4*>(optr + 32 * cc);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        dst[i] = make_uint4(o16[4 * i], o16[4 * i + 1], o16[4 * i + 2], o16[4 * i + 3]);
+                        for (int i = 0; i < 4; ++i)
+                            dst[i] = make_uint4(o16[4 * i], o16[4 * i + 1], o16[4 * i + 2], o16[4 * i + 3]);
+                    }
                 }
             }
-            if (valid && wg == 0 && p.lse) p.lse[orow] = finalize_lse(M_g, Ltot, c);
         }
     }
 
