@@ -384,7 +384,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         m_old = st_m[r];
                     }
                 }
-                const float m_new = fmaxf(m_old, mt);
+                const float m_new = softmax_next_max(m_old, mt, c);
                 st_m[r] = m_new;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_m);

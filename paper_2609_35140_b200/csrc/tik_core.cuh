@@ -16,7 +16,9 @@
 //   * c = softmax_scale * log2(e), one fp32 multiply on the host.
 //   * Mask: select -inf where key position > query position (no arithmetic on masked
 //     scores, so masked K contents never matter).
-//   * Per tile and row: m' = max(m, tile max); p = ex2.approx.ftz(fma(s, c, -(m' * c)));
+//   * Per tile and row: the reference m moves to the tile maximum only when that exceeds it
+//     by more than 8 in the exponent, (tile max - m) * c > 8 (so always on the first tile of
+//     a chunk), else m' = m; p = ex2.approx.ftz(fma(s, c, -(m' * c)));
 //     row sums in the fixed two-halves-of-four-chains shape below; alpha = ex2.approx.ftz((m - m') * c);
 //     l_half = fma(l_half, alpha, rowsum of that 64-column half); O = O * alpha with a non-flushing IEEE multiply (so
 //     skipping it when alpha == 1.0f is bit-neutral); P rounded to bf16 (RNE) for the PV
@@ -38,7 +40,7 @@ constexpr float LN2_F = 0.69314718055994530942f;
 constexpr int LP_TILE = 128;          // vocabulary columns per log-sum-exp tile
 constexpr int LP_SUPER = 1024;        // vocabulary columns per super-chunk (8 tiles)
 
-#define TIK_CONTRACT_ID "tik2-BN128-CH2048-M128N128K16-ex2ftz-sum2x4-LP128x1024"
+#define TIK_CONTRACT_ID "tik3-BN128-CH2048-M128N128K16-ex2ftz-lazy8-sum2x4-LP128x1024"
 
 __device__ __forceinline__ float ex2_ftz(float x) {
     float y;
@@ -86,6 +88,17 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float y;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
     return y;
+}
+
+// Reference maximum after a tile whose (masked) maximum is mt.  The reference only moves when
+// the tile maximum exceeds it by more than 2^RESCALE_LOG2 in the exponent (always on the first
+// tile of a chunk, where it is -inf); otherwise it stays, weights may reach 2^RESCALE_LOG2
+// instead of 1, alpha is exactly 1 and the accumulator is not rescaled.  The decision reads
+// only the row's own scores and the fixed tile boundaries, so it is the same in every regime.
+constexpr float RESCALE_LOG2 = 8.0f;
+__device__ __forceinline__ float softmax_next_max(float m_ref, float mt, float c) {
+    const float growth = __fmul_rn(__fsub_rn(mt, m_ref), c);
+    return (growth > RESCALE_LOG2) ? mt : m_ref;
 }
 
 // exponent argument of one score: s * c - mc, one fused multiply-add.
