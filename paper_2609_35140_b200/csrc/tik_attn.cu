@@ -194,6 +194,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             }
             const CUtensorMap* tm = kv ? &tmV : &tmK;
             for (int it = 0; it < n_tiles; ++it) {
+                if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
                 const int j = tile_first + it;
                 const int st = it % KV_STAGES;
                 const uint32_t use = it / KV_STAGES;
@@ -243,6 +244,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             mbar_wait(bar_q, 0, abort_word, p.dev_status);
             const uint64_t dq = smem_desc_sw128(sQ, 0, 1024);
             for (int x = 0; x < n_tiles; ++x) {
+                if (*abort_word) break;
                 const int st = x % KV_STAGES, b = x & 1;
                 // the single score buffer is free once the softmax of tile x-1 holds it in registers
                 if (x >= 1) mbar_wait(bar_sempty + 8 * ((x - 1) & 1), ((x - 1) >> 1) & 1, abort_word, p.dev_status);
@@ -260,6 +262,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // ------------------------------------------------------------ PV issuer
         if (lane == 0) {
             for (int x = 0; x < n_tiles; ++x) {
+                if (*abort_word) break;
                 const int st = x % KV_STAGES, b = x & 1;
                 mbar_wait(bar_vfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
                 mbar_wait(bar_pfull + 8 * b, (x >> 1) & 1, abort_word, p.dev_status);
@@ -336,6 +339,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         const int last = n_tiles - 1;
 
         for (int it = wg; it < n_tiles; it += 2) {
+            if (*abort_word) break;
             const int j = tile_first + it;
             const bool chunk_start = is_chunk_start(it);
             mbar_wait(bar_sfull + 8 * wg, (it >> 1) & 1, abort_word, p.dev_status);
@@ -393,24 +397,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 RowSum4 rs_lo, rs_hi;
                 rs_lo.reset();
                 rs_hi.reset();
+                // a masked score is -inf: the fma gives -inf and ex2 gives +0 exactly
 #pragma unroll
-                for (int i = 0; i < 64; i += 2) {
-                    // a masked score is -inf: fma gives -inf and ex2 gives +0 exactly
-                    const float p0 = softmax_p(__uint_as_float(sc[i]), c, neg_mc);
-                    const float p1 = softmax_p(__uint_as_float(sc[i + 1]), c, neg_mc);
-                    rowsum_add(rs_lo, i, p0);
-                    rowsum_add(rs_lo, i + 1, p1);
-                    sc[i >> 1] = pack_bf16x2(p0, p1);
-                }
+                for (int i = 0; i < 64; i += 8) softmax_p8(&sc[i], c, neg_mc, rs_lo, &sc[i >> 1]);
                 tmem_st32(tp, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
 #pragma unroll
-                for (int i = 0; i < 64; i += 2) {
-                    const float p0 = softmax_p(__uint_as_float(sc[64 + i]), c, neg_mc);
-                    const float p1 = softmax_p(__uint_as_float(sc[64 + i + 1]), c, neg_mc);
-                    rowsum_add(rs_hi, i, p0);
-                    rowsum_add(rs_hi, i + 1, p1);
-                    sc[32 + (i >> 1)] = pack_bf16x2(p0, p1);
-                }
+                for (int i = 0; i < 64; i += 8) softmax_p8(&sc[64 + i], c, neg_mc, rs_hi, &sc[32 + (i >> 1)]);
                 tmem_st32(tp + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[32]));
                 if (it > 0 && !fold_now) {
                     mbar_wait(bar_l, (it - 1) & 1, abort_word, p.dev_status);
@@ -525,9 +517,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     }
 
     // ---------------------------------------------------------------- teardown
-    if (*abort_word) {   // let copies in flight land before the CTA's shared memory is released
+    if (*abort_word) {   // let copies and MMAs in flight finish before shared memory and TMEM are released
         const unsigned long long t0 = globaltimer_ns();
-        while (globaltimer_ns() - t0 < 200000ull) {
+        while (globaltimer_ns() - t0 < 1000000ull) {
         }
     }
     tc_fence_before();

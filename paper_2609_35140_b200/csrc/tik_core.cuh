@@ -101,6 +101,44 @@ __device__ __forceinline__ float softmax_next_max(float m_ref, float mt, float c
     return (growth > RESCALE_LOG2) ? mt : m_ref;
 }
 
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits), RNE
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+
+// Two-wide forms of the same IEEE operations (fma.rn / add.rn on f32 pairs): identical bits to
+// the scalar intrinsics, half the issue slots.
+__device__ __forceinline__ void fma_rn_x2(float& d0, float& d1, float a0, float a1, float b, float c) {
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+__device__ __forceinline__ void add_rn_x2(float& a0, float& a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb;\n\t"
+        "mov.b64 ra, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\t"
+        "add.rn.f32x2 ra, ra, rb;\n\tmov.b64 {%0, %1}, ra;\n\t}"
+        : "+f"(a0), "+f"(a1)
+        : "f"(b0), "f"(b1));
+}
+// Weights and half-row sum of 8 consecutive columns (chains 0,0,1,1,2,2,3,3): every chain still
+// receives its columns in ascending order, two chains per packed add.
+__device__ __forceinline__ void softmax_p8(const uint32_t* s8, float c, float neg_mc, RowSum4& rs, uint32_t* pk4) {
+    float x[8];
+#pragma unroll
+    for (int i = 0; i < 8; i += 2)
+        fma_rn_x2(x[i], x[i + 1], __uint_as_float(s8[i]), __uint_as_float(s8[i + 1]), c, neg_mc);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = ex2_ftz(x[i]);
+    add_rn_x2(rs.a[0], rs.a[1], x[0], x[2]);
+    add_rn_x2(rs.a[2], rs.a[3], x[4], x[6]);
+    add_rn_x2(rs.a[0], rs.a[1], x[1], x[3]);
+    add_rn_x2(rs.a[2], rs.a[3], x[5], x[7]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) pk4[i] = pack_bf16x2(x[2 * i], x[2 * i + 1]);
+}
+
 // exponent argument of one score: s * c - mc, one fused multiply-add.
 __device__ __forceinline__ float softmax_p(float s, float c, float neg_mc) {
     return ex2_ftz(__fmaf_rn(s, c, neg_mc));
@@ -112,10 +150,6 @@ __device__ __forceinline__ float softmax_alpha(float m_old, float m_new, float c
 }
 __device__ __forceinline__ float rescale_o(float o, float alpha) { return __fmul_rn(o, alpha); }
 
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits), RNE
-    return *reinterpret_cast<uint32_t*>(&t);
-}
 
 // Fold chunk state (m_c, l_c, O_c) into the global state (M, L, O).  The global state is
 // initialised by copying chunk 0; chunks 1, 2, ... are folded in ascending order.

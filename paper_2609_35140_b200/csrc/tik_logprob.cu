@@ -94,6 +94,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int nt = 0; nt < n_nt; ++nt) {
                 const int col0 = col_base + nt * LP_TILE;
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
                     const int s = it % STAGES;
                     const uint32_t use = it / STAGES;
                     if (use > 0) mbar_wait(bar_empty + 8 * s, (use - 1) & 1, abort_word, p.dev_status);
@@ -113,6 +114,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (use > 0) mbar_wait(bar_acc_empty + 8 * buf, (use - 1) & 1, abort_word, p.dev_status);
                 tc_fence_after();
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    if (*abort_word) break;
                     const int s = it % STAGES;
                     mbar_wait(bar_full + 8 * s, (it / STAGES) & 1, abort_word, p.dev_status);
                     tc_fence_after();
@@ -194,7 +196,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (*abort_word) {
         const unsigned long long t0 = globaltimer_ns();
-        while (globaltimer_ns() - t0 < 200000ull) {
+        while (globaltimer_ns() - t0 < 1000000ull) {
         }
     }
     tc_fence_before();
