@@ -1,0 +1,125 @@
+"""Full-size parity: the benchmark workloads at their real sizes, in the launch configuration
+bench.py times.  The oracle checks sampled rows one by one; the cross-regime comparison is exact
+on every row it touches (prefill rows of every prompt, decode rows at sampled positions)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_35140_b200 import synth
+from gpu_common import ATTN_TOL, LOGPROB_TOL, count_diff
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tik():
+    from paper_2609_35140_b200 import binding
+    binding.load()
+    yield binding
+    assert binding.device_status() == 0
+
+
+def _oracle_rows(w, q, k, v, rows):
+    """Oracle outputs for (sequence, head, position) rows, copying only the K/V slices they need."""
+    cu = w.cu_seqlens()
+    ks, vs, qs, off, ln = [], [], [], [], []
+    base = 0
+    cache = {}
+    for (s, h, t) in rows:
+        g = h // w.G
+        if (s, g) not in cache:
+            sl = slice(int(cu[s]), int(cu[s + 1]))
+            ks.append(k[sl, g].float().cpu().numpy())
+            vs.append(v[sl, g].float().cpu().numpy())
+            cache[(s, g)] = base
+            base += w.seq_lens[s]
+        qs.append(q[int(cu[s]) + t, h].float().cpu().numpy())
+        off.append(cache[(s, g)])
+        ln.append(t + 1)
+    out, _ = oracle.attn_rows(np.stack(qs), np.concatenate(ks), np.concatenate(vs), off, ln, w.softmax_scale)
+    return out
+
+
+@pytest.mark.parametrize("index", [1, 2, 3, 4])
+def test_attention_at_full_size(tik, index):
+    w = synth.get_workload(index)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    cu_h = w.cu_seqlens()
+    o_train = tik.tik_attn_train_fwd(q, k, v, cu, max(w.seq_lens), w.softmax_scale)
+
+    # --- oracle on sampled rows (boundaries of tiles, pages and chunks, first/last rows, random)
+    rng = np.random.default_rng(w.seed + 17)
+    seqs = sorted(set([int(np.argmin(w.seq_lens)), int(np.argmax(w.seq_lens))] +
+                      [int(x) for x in rng.integers(0, w.S, 2)]))
+    rows = []
+    for s in seqs:
+        L = w.seq_lens[s]
+        marks = [0, 1, 63, 64, 127, 128, 129, w.prompt_lens[s] - 1, w.prompt_lens[s], 2047, 2048, 2049,
+                 4095, 4096, L // 2, L - 2, L - 1] + [int(x) for x in rng.integers(0, L, 6)]
+        for t in marks:
+            if 0 <= t < L:
+                rows.append((s, int(rng.integers(0, w.Hq)), t))
+    ref = _oracle_rows(w, q, k, v, rows)
+    got = torch.stack([o_train[int(cu_h[s]) + t, h] for (s, h, t) in rows]).float().cpu().numpy()
+    assert np.abs(got - ref).max() <= ATTN_TOL
+    del ref, got
+
+    # --- rollout: cache write, prefill of one prompt per group, decode at sampled positions
+    layout = synth.make_paged_layout(w)
+    bt = torch.from_numpy(layout.block_table).cuda()
+    kc = torch.zeros(layout.num_pages, w.Hkv, layout.page_size, w.d, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    firsts = sorted({g: s for s, g in reversed(list(enumerate(w.group_of)))}.values())
+    prow = torch.cat([torch.arange(cu_h[s], cu_h[s] + w.prompt_lens[s]) for s in firsts]).cuda()
+    plens = [w.prompt_lens[s] for s in firsts]
+    cu_q = torch.tensor(np.concatenate([[0], np.cumsum(plens)]), dtype=torch.int32, device="cuda")
+    pctx = torch.tensor(plens, dtype=torch.int32, device="cuda")
+    pbt = bt[firsts].contiguous()
+    tik.tik_kv_cache_write(k[prow].contiguous(), v[prow].contiguous(), cu_q, pctx, kc, vc, pbt)
+    o_pre = tik.tik_attn_prefill(q[prow].contiguous(), cu_q, pctx, kc, vc, pbt, max(plens), max(plens),
+                                 w.softmax_scale)
+    assert count_diff(o_pre, o_train[prow]) == 0
+    del o_pre
+    # the rest of every sequence goes into the cache (shared prompt pages are rewritten with equal data)
+    ctx_full = torch.tensor(w.seq_lens, dtype=torch.int32, device="cuda")
+    tik.tik_kv_cache_write(k, v, cu, ctx_full, kc, vc, bt)
+    all_seqs = list(range(w.S))
+    ws = torch.empty(tik.workspace_bytes(tik.OP_ATTN_DECODE, w.S, w.Hq, w.Hkv, w.d, max(w.seq_lens)),
+                     dtype=torch.uint8, device="cuda")
+    points = [1.0, 0.5] + ([c for c in (w.decode_contexts or [])])
+    for pt in points:
+        if pt <= 1.0:
+            pos = [max(w.prompt_lens[s], int(w.seq_lens[s] * pt)) - 1 for s in all_seqs]
+        else:
+            pos = [min(int(pt), w.seq_lens[s]) - 1 for s in all_seqs]
+        drow = torch.tensor([int(cu_h[s]) + p for s, p in zip(all_seqs, pos)], device="cuda")
+        ctx = torch.tensor([p + 1 for p in pos], dtype=torch.int32, device="cuda")
+        o_dec = tik.tik_attn_decode(q[drow].contiguous(), ctx, kc, vc, bt, max(pos) + 1, w.softmax_scale, ws=ws)
+        assert count_diff(o_dec, o_train[drow]) == 0, pt
+    # a single sequence decoded alone gives the same bits as inside the full batch
+    s = seqs[-1]
+    p1 = w.seq_lens[s] - 1
+    o1 = tik.tik_attn_decode(q[int(cu_h[s]) + p1][None].contiguous(), torch.tensor([p1 + 1], dtype=torch.int32,
+                             device="cuda"), kc, vc, bt[s][None].contiguous(), p1 + 1, w.softmax_scale)
+    assert count_diff(o1[0], o_train[int(cu_h[s]) + p1]) == 0
+
+
+@pytest.mark.parametrize("index", [1, 2, 3, 4])
+def test_logprob_at_full_size(tik, index):
+    w = synth.get_workload(index)
+    hidden, W, target = synth.make_logprob_inputs(w, "cuda")
+    T = hidden.shape[0]
+    lp = tik.tik_token_logprob(hidden, W, target)
+    rng = np.random.default_rng(w.seed + 23)
+    n = 48 if index <= 2 else 24
+    sample = np.unique(np.concatenate([[0, 127, 128, T - 1], rng.integers(0, T, n)]))
+    st = torch.from_numpy(sample).cuda()
+    ref, _ = oracle.token_logprob(hidden[st].float().cpu().numpy(), W.float().cpu().numpy(),
+                                  target[st].cpu().numpy())
+    assert np.abs(lp[st].cpu().numpy() - ref).max() <= LOGPROB_TOL
+    assert bool(torch.isfinite(lp).all())
+    # decode-shaped and prefill-shaped calls over the same rows give identical bits
+    for a, b in [(0, 1), (0, w.S), (T - 300, T), (1000, 1000 + 64)]:
+        part = tik.tik_token_logprob(hidden[a:b].contiguous(), W, target[a:b].contiguous())
+        assert count_diff(part, lp[a:b]) == 0, (a, b)
