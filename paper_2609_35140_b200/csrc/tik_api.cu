@@ -344,8 +344,9 @@ tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_he
     uint64_t bd[2] = {static_cast<uint64_t>(H), static_cast<uint64_t>(V)};
     uint64_t st1[1] = {static_cast<uint64_t>(H) * 2};
     uint32_t box[2] = {64, 128};
+    uint32_t boxB[2] = {64, 256};        // 256 vocabulary rows per MMA step
     if (!make_tmap_bf16(ctx, &tmA, hidden, 2, ad, st1, box, &err) ||
-        !make_tmap_bf16(ctx, &tmB, lm_head, 2, bd, st1, box, &err))
+        !make_tmap_bf16(ctx, &tmB, lm_head, 2, bd, st1, boxB, &err))
         return fail(ctx, TIK_ERR_CUDA, err.c_str());
 
     LogprobParams p{};

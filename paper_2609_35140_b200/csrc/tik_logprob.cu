@@ -2,13 +2,14 @@
 // log-sum-exp over the vocabulary and the target-logit gather.  The fp32 logits live only
 // in TMEM; nothing of size T x V is ever written.
 //
-// One CTA = (128-token tile, 1024-column super-chunk).  For each of the (up to) eight
-// 128-column tiles of the super-chunk, a TMA warp streams 64-wide K slices of hidden and
+// One CTA = (128-token tile, 1024-column super-chunk).  For each of the (up to) four
+// 256-column steps of the super-chunk, a TMA warp streams 64-wide K slices of hidden and
 // lm_head through a shared-memory ring, an MMA warp accumulates the whole K range in
-// ascending order into one of two TMEM accumulators (no split-K), and four epilogue warps
-// (one thread per token row) reduce the finished tile to (max, sum of exp) with the fixed
-// row-sum shape, fold it into the super-chunk's running pair, and pick the target logit if
-// this tile owns its column.  A finish kernel folds the super-chunk pairs of every token in
+// ascending order into one of two 256-column TMEM accumulators (M128 x N256 x K16 MMAs, no
+// split-K), and four epilogue warps (one thread per token row) reduce each of its two
+// 128-column tiles to (max, sum of exp) with the fixed row-sum shape, fold them in ascending
+// order into the super-chunk's running pair, and pick the target logit if a tile owns its
+// column.  A finish kernel folds the super-chunk pairs of every token in
 // ascending order and writes logprob = z_target - logsumexp.
 #include "tik_core.cuh"
 #include "tik_internal.h"
@@ -17,9 +18,10 @@
 namespace tik {
 
 namespace lp {
-constexpr int STAGES = 6;
+constexpr int STAGES = 4;
+constexpr int NB = 256;                      // vocabulary columns per MMA (two log-sum-exp tiles)
 constexpr uint32_t A_BYTES = 128 * 128;      // 128 token rows x 64 bf16
-constexpr uint32_t B_BYTES = 128 * 128;      // 128 vocab rows x 64 bf16
+constexpr uint32_t B_BYTES = NB * 128;       // 256 vocab rows x 64 bf16
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr uint32_t OFF_BAR = STAGES * STAGE_BYTES;
 constexpr uint32_t BYTES = OFF_BAR + 256;
@@ -32,8 +34,8 @@ __global__ void __launch_bounds__(lp::THREADS, 1)
 logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const LogprobParams p) {
     using namespace lp;
-    constexpr uint32_t TMEM_COLS = 256;      // two 128-column accumulators
-    constexpr uint32_t IDESC = mma_idesc_bf16(128, 128, false);
+    constexpr uint32_t TMEM_COLS = 512;      // two 256-column accumulators
+    constexpr uint32_t IDESC = mma_idesc_bf16(128, NB, false);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // raster: bands of BAND token tiles; within a band the token tile varies fastest so the
@@ -49,7 +51,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (tile_in_band >= band_tiles) return;
     const int tok0 = (band * BAND + tile_in_band) * 128;
     const int col_base = sup * LP_SUPER;
-    const int n_nt = min(LP_SUPER / LP_TILE, (p.V - col_base + LP_TILE - 1) / LP_TILE);
+    const int n_nt = min(LP_SUPER / NB, (p.V - col_base + NB - 1) / NB);   // 256-column steps
     const int n_kb = p.H / 64;
 
     extern __shared__ uint8_t smem_raw[];
@@ -92,7 +94,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             uint32_t it = 0;
             for (int nt = 0; nt < n_nt; ++nt) {
-                const int col0 = col_base + nt * LP_TILE;
+                const int col0 = col_base + nt * NB;
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
                     const int s = it % STAGES;
@@ -119,7 +121,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     mbar_wait(bar_full + 8 * s, (it / STAGES) & 1, abort_word, p.dev_status);
                     tc_fence_after();
                     const uint32_t a0 = sbase + s * STAGE_BYTES, b0 = a0 + A_BYTES;
-                    mma_ss_chain4(tmem + buf * 128, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
+                    mma_ss_chain4(tmem + buf * NB, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
                                   IDESC, kb ? 1u : 0u);
                     mma_commit(bar_empty + 8 * s);
                 }
@@ -135,58 +137,64 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int target = row_valid ? p.target[t] : -1;
         const float it_scale = p.inv_temperature;
         float M = -CUDART_INF_F, Lsum = 0.0f;
+        bool first = true;
         for (int nt = 0; nt < n_nt; ++nt) {
             const int buf = nt & 1;
-            const int col0 = col_base + nt * LP_TILE;
             mbar_wait(bar_acc_full + 8 * buf, (nt >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
-            const uint32_t taddr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 128;
-            const int vmax = p.V - 1 - col0;               // columns > vmax are past the vocabulary
-            float mt = -CUDART_INF_F;
+#pragma unroll 1
+            for (int half = 0; half < NB / LP_TILE; ++half) {
+                const int col0 = col_base + nt * NB + half * LP_TILE;
+                if (col0 >= p.V) break;                        // tile entirely past the vocabulary
+                const uint32_t taddr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * NB + half * LP_TILE;
+                const int vmax = p.V - 1 - col0;               // columns > vmax are past the vocabulary
+                float mt = -CUDART_INF_F;
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t v[32];
-                tmem_ld32(taddr + 32 * cc, v);
-                tmem_wait_ld();
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + 32 * cc, v);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float z = __fmul_rn(__uint_as_float(v[i]), it_scale);
-                    if (32 * cc + i > vmax) z = -CUDART_INF_F;
-                    mt = fmaxf(mt, z);
+                    for (int i = 0; i < 32; ++i) {
+                        float z = __fmul_rn(__uint_as_float(v[i]), it_scale);
+                        if (32 * cc + i > vmax) z = -CUDART_INF_F;
+                        mt = fmaxf(mt, z);
+                    }
                 }
-            }
-            const float neg_mc = -__fmul_rn(mt, LOG2E_F);
-            const int tcol = target - col0;                // in [0,128) when this tile owns the target
-            float zt = 0.0f;
-            RowSum8 rs;
-            rs.reset();
+                const float neg_mc = -__fmul_rn(mt, LOG2E_F);
+                const int tcol = target - col0;                // in [0,128) when this tile owns the target
+                float zt = 0.0f;
+                RowSum8 rs;
+                rs.reset();
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t v[32];
-                tmem_ld32(taddr + 32 * cc, v);
-                tmem_wait_ld();
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + 32 * cc, v);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float z = __fmul_rn(__uint_as_float(v[i]), it_scale);
-                    float e = softmax_p(z, LOG2E_F, neg_mc);
-                    if (32 * cc + i > vmax) e = 0.0f;
-                    rowsum_add(rs, 32 * cc + i, e);
-                    if (32 * cc + i == tcol) zt = z;
+                    for (int i = 0; i < 32; ++i) {
+                        const float z = __fmul_rn(__uint_as_float(v[i]), it_scale);
+                        float e = softmax_p(z, LOG2E_F, neg_mc);
+                        if (32 * cc + i > vmax) e = 0.0f;
+                        rowsum_add(rs, 32 * cc + i, e);
+                        if (32 * cc + i == tcol) zt = z;
+                    }
                 }
+                const float lt = rs.total();
+                if (first) {
+                    M = mt;
+                    Lsum = lt;
+                    first = false;
+                } else {
+                    const FoldCoef f = fold_coef(M, mt, LOG2E_F);
+                    Lsum = fold_value(Lsum, lt, f);
+                    M = f.M_new;
+                }
+                if (row_valid && tcol >= 0 && tcol < LP_TILE && target < p.V) p.z_target[t] = zt;
             }
             // all TMEM reads of this accumulator are done: hand it back to the MMA warp
             tc_fence_before();
             mbar_arrive(bar_acc_empty + 8 * buf);
-            const float lt = rs.total();
-            if (nt == 0) {
-                M = mt;
-                Lsum = lt;
-            } else {
-                const FoldCoef f = fold_coef(M, mt, LOG2E_F);
-                Lsum = fold_value(Lsum, lt, f);
-                M = f.M_new;
-            }
-            if (row_valid && tcol >= 0 && tcol < LP_TILE && target < p.V) p.z_target[t] = zt;
         }
         if (row_valid) {
             p.part_ml[2 * (t * p.nsuper + sup)] = M;
