@@ -127,7 +127,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const uint32_t bar_sfull = bar0 + 136;       // [2] QK^T of an even / odd tile done: scores ready in TMEM
     const uint32_t bar_pfull = bar0 + 152;       // [2] P written over the scores, O rescaled (4 warps)
     const uint32_t bar_pempty = bar0 + 168;      // [2] PV done: O updated, weight buffer free
-    const uint32_t bar_hand = bar0 + 184;        // [2][4] row-state hand-off between the warpgroups
+    const uint32_t bar_hand = bar0 + 184;        // [4] reference-maximum hand-off between the warpgroups
     const uint32_t bar_sempty = bar0 + 248;      // [2] scores of a tile are in registers (4 warps)
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 264);
     volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 268);
@@ -147,7 +147,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             mbar_init(bar_sempty + 8 * i, 4);
             mbar_init(bar_pempty + 8 * i, 1);
         }
-        for (int i = 0; i < 8; ++i) mbar_init(bar_hand + 8 * i, 1);
+        for (int i = 0; i < 4; ++i) mbar_init(bar_hand + 8 * i, 1);
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmQ);
@@ -244,7 +244,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             mbar_wait(bar_q, 0, abort_word, p.dev_status);
             const uint64_t dq = smem_desc_sw128(sQ, 0, 1024);
             for (int x = 0; x < n_tiles; ++x) {
-                if (*abort_word) break;
                 const int st = x % KV_STAGES, b = x & 1;
                 // the single score buffer is free once the softmax of tile x-1 holds it in registers
                 if (x >= 1) mbar_wait(bar_sempty + 8 * ((x - 1) & 1), ((x - 1) >> 1) & 1, abort_word, p.dev_status);
@@ -262,7 +261,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // ------------------------------------------------------------ PV issuer
         if (lane == 0) {
             for (int x = 0; x < n_tiles; ++x) {
-                if (*abort_word) break;
                 const int st = x % KV_STAGES, b = x & 1;
                 mbar_wait(bar_vfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
                 mbar_wait(bar_pfull + 8 * b, (x >> 1) & 1, abort_word, p.dev_status);
@@ -283,8 +281,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // While one warpgroup is in its exp2 phase the other loads scores, reduces the maximum
         // and stores weights, so the special-function unit stays busy.  The row state (running
         // maximum, the two half row sums, the folded state of earlier chunks) lives in shared
-        // memory and is handed from the thread of tile it to the thread of tile it+1 through
-        // two mbarriers per lane quarter.
+        // memory and is handed from the thread of tile it to the thread of tile it+1: the maximum
+        // through an mbarrier per lane quarter, the row sums with the "weights written" barrier.
         const int wg = (warp - 4) >> 2;
         const int quarter = warp & 3;                       // TMEM lane quarter of this warp
         const int r = quarter * 32 + lane;                  // tile row == TMEM lane
@@ -295,7 +293,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         float* st_m = lx;                 // [128]    running maximum of the current chunk
         float* st_l = lx + 128;           // [2][128] half row sums of the current chunk
         const uint32_t bar_m = bar_hand + 8 * quarter;       // "maximum of tile it published"
-        const uint32_t bar_l = bar_hand + 32 + 8 * quarter;  // "row sums of tile it published"
         const uint32_t ts = tlane + COL_S;
         const uint32_t tp = tlane + COL_P + 64 * wg;
         // Folded state of the finished chunks.  Both threads of a row keep it: warpgroup 0 folds
@@ -307,6 +304,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         auto wait_pv = [&](int x) {
             mbar_wait(bar_pempty + 8 * (x & 1), (x >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
+        };
+        // The other warpgroup has finished tile x (weights and row sums written): the barrier the
+        // PV issuer waits on doubles as the hand-off of the row sums.
+        auto wait_tile_done = [&](int x) {
+            mbar_wait(bar_pfull + 8 * (x & 1), (x >> 1) & 1, abort_word, p.dev_status);
         };
         // folds a finished chunk (m_c, l_c halves) into the global row state; with_o also folds
         // its accumulator O_B into O_A (one thread per row does that, after the chunk's last PV)
@@ -339,7 +341,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         const int last = n_tiles - 1;
 
         for (int it = wg; it < n_tiles; it += 2) {
-            if (*abort_word) break;
             const int j = tile_first + it;
             const bool chunk_start = is_chunk_start(it);
             mbar_wait(bar_sfull + 8 * wg, (it >> 1) & 1, abort_word, p.dev_status);
@@ -365,14 +366,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     for (int i = 0; i < 128; ++i)
                         if (i > kmax) sc[i] = 0xff800000u;          // -inf
                 }
-                float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+                float mx[8];
 #pragma unroll
-                for (int i = 0; i < 128; i += 8) {
+                for (int k = 0; k < 8; ++k) mx[k] = fmaxf(__uint_as_float(sc[2 * k]), __uint_as_float(sc[2 * k + 1]));
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
+                for (int i = 16; i < 128; i += 16) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
                         mx[k] = fmax3(mx[k], __uint_as_float(sc[i + 2 * k]), __uint_as_float(sc[i + 2 * k + 1]));
                 }
-                const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                const float mt = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmax3(fmax3(mx[3], mx[4], mx[5]), mx[6], mx[7]));
                 // state handed over by the thread that processed tile it-1
                 float m_old = -CUDART_INF_F, l_old_lo = 0.0f, l_old_hi = 0.0f;
                 float m_prev = 0.0f, l_prev_lo = 0.0f, l_prev_hi = 0.0f;   // finished chunk, if any
@@ -380,7 +383,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 if (it > 0) {
                     mbar_wait(bar_m, (it - 1) & 1, abort_word, p.dev_status);
                     if (fold_now) {
-                        mbar_wait(bar_l, (it - 1) & 1, abort_word, p.dev_status);
+                        wait_tile_done(it - 1);
                         m_prev = st_m[r];
                         l_prev_lo = st_l[r];
                         l_prev_hi = st_l[128 + r];
@@ -405,7 +408,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 for (int i = 0; i < 64; i += 8) softmax_p8(&sc[64 + i], c, neg_mc, rs_hi, &sc[32 + (i >> 1)]);
                 tmem_st32(tp + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[32]));
                 if (it > 0 && !fold_now) {
-                    mbar_wait(bar_l, (it - 1) & 1, abort_word, p.dev_status);
+                    wait_tile_done(it - 1);
                     if (!chunk_start) {
                         l_old_lo = st_l[r];
                         l_old_hi = st_l[128 + r];
@@ -444,7 +447,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             if (lane == 0) {
                 if (!active) mbar_arrive(bar_sempty + 8 * wg);
                 mbar_arrive(bar_pfull + 8 * wg);
-                if (active) mbar_arrive(bar_l);
             }
         }
 
