@@ -180,56 +180,71 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // ------------------------------------------------------------ TMA producers
         // warp 0 streams Q and the K tiles, warp 2 the V tiles: a K tile is requested as soon as
         // the QK^T that used its stage has finished, without queueing behind a wait for PV.
-        if (lane == 0) {
-            const int kv = (warp == 2) ? 1 : 0;
-            if (kv == 0) {
-                if (MODE == MODE_DECODE) {
-                    mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
-                    for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
-                } else {
-                    mbar_expect_tx(bar_q, L::TILE);
-                    for (int a = 0; a < NATOM; ++a)
-                        tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
+        const int kv = (warp == 2) ? 1 : 0;
+        const CUtensorMap* tm = kv ? &tmV : &tmK;
+        if (kv == 0 && lane == 0) {
+            if (MODE == MODE_DECODE) {
+                mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
+                for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
+            } else {
+                mbar_expect_tx(bar_q, L::TILE);
+                for (int a = 0; a < NATOM; ++a)
+                    tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
+            }
+        }
+        if (MODE == MODE_TRAIN) {
+            if (lane == 0) {
+                for (int it = 0; it < n_tiles; ++it) {
+                    if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
+                    const int st = it % KV_STAGES;
+                    const uint32_t use = it / KV_STAGES;
+                    const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
+                    const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
+                    // Each stage has its own release barrier with this thread as its only waiter: a
+                    // barrier shared with waiters of a different lag could run two phases ahead of
+                    // the slowest one, which a parity wait cannot tell from "not yet".
+                    if (use > 0)
+                        mbar_wait((kv ? bar_vempty : bar_kempty) + 8 * st, (use - 1) & 1, abort_word, p.dev_status);
+                    mbar_expect_tx(full, L::TILE);
+                    const int row = static_cast<int>(tok0) + 128 * (tile_first + it);
+                    for (int a = 0; a < NATOM; ++a) tma_load_3d(dst + a * L::ATOM, tm, full, a * 64, kvh, row);
                 }
             }
-            const CUtensorMap* tm = kv ? &tmV : &tmK;
+        } else {
+            // Paged K/V: the warp reads 32 block-table entries at a time (one per lane, coalesced),
+            // so the table's latency is paid once per 32 pages instead of before every tile.
+            const int ppt = p.pages_per_tile;
+            const int tiles_per_batch = 32 / ppt;
+            int my_phys = p.num_pages;
             for (int it = 0; it < n_tiles; ++it) {
-                if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
+                if (*abort_word) break;
                 const int j = tile_first + it;
+                const int in_batch = it % tiles_per_batch;
+                if (in_batch == 0) {
+                    const int lp = (128 * j) / p.page_size + lane;
+                    int ph = p.num_pages;       // out of range: the box is filled with zeros
+                    if (lp * p.page_size < ctx) {
+                        ph = (lp < p.max_blocks) ? p.block_table[static_cast<long long>(seq) * p.max_blocks + lp] : -1;
+                        if (ph < 0 || ph >= p.num_pages) {
+                            if (kv == 0) atomicOr(p.dev_status, TIK_DEV_BAD_BLOCK);
+                            ph = p.num_pages;
+                        }
+                    }
+                    my_phys = ph;
+                }
                 const int st = it % KV_STAGES;
                 const uint32_t use = it / KV_STAGES;
                 const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
                 const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
-                int phys[8];
-                if (MODE != MODE_TRAIN) {
-                    const int lp0 = (128 * j) / p.page_size;
-                    for (int i = 0; i < p.pages_per_tile; ++i) {
-                        const int lp = lp0 + i;
-                        int ph = p.num_pages;   // out of range: the box is filled with zeros
-                        if (lp * p.page_size < ctx) {
-                            ph = (lp < p.max_blocks) ? p.block_table[static_cast<long long>(seq) * p.max_blocks + lp] : -1;
-                            if (ph < 0 || ph >= p.num_pages) {
-                                atomicOr(p.dev_status, TIK_DEV_BAD_BLOCK);
-                                ph = p.num_pages;
-                            }
-                        }
-                        phys[i] = ph;
-                    }
-                }
-                // Each stage has its own release barrier with this thread as its only waiter: a
-                // barrier shared with waiters of a different lag could run two phases ahead of
-                // the slowest one, which a parity wait cannot tell from "not yet".
                 if (use > 0)
                     mbar_wait((kv ? bar_vempty : bar_kempty) + 8 * st, (use - 1) & 1, abort_word, p.dev_status);
-                mbar_expect_tx(full, L::TILE);
-                if (MODE == MODE_TRAIN) {
-                    const int row = static_cast<int>(tok0) + 128 * j;
-                    for (int a = 0; a < NATOM; ++a) tma_load_3d(dst + a * L::ATOM, tm, full, a * 64, kvh, row);
-                } else {
-                    for (int i = 0; i < p.pages_per_tile; ++i) {
+                if (lane == 0) mbar_expect_tx(full, L::TILE);
+                for (int i = 0; i < ppt; ++i) {
+                    const int phys = __shfl_sync(0xffffffffu, my_phys, in_batch * ppt + i);
+                    if (lane == 0) {
                         const uint32_t off = static_cast<uint32_t>(i * p.page_size) * 128u;
                         for (int a = 0; a < NATOM; ++a)
-                            tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, phys[i]);
+                            tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, phys);
                     }
                 }
             }
