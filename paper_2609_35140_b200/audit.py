@@ -1,0 +1,201 @@
+"""Evaluation-specification harness for the attention kernels (paper Sec. 4.1 and 5.2).
+
+The paper promotes a kernel revision only if it is *verified* (all prescribed correctness checks
+pass), *admissible* (every workload of a fixed set stays within a per-workload slowdown limit of a
+recorded baseline) and has a strictly lower weighted sum of workload latencies
+T = sum_w c_w * lat(w) (Eq. 2).  This module is that rule for this repository:
+
+  * workloads: the paper's per-operator grid (Sec. 6 Q3) -- prefill of 1K/4K/8K/16K tokens at
+    batch 1, decode at context 128/1K/4K/8K x batch 1/4/8/16 -- with the long-context head
+    shape (32 query heads, 8 KV heads, head_dim 128, page 64), unit weights;
+  * correctness: entry-point consistency (prefill rows and decode rows equal the packed
+    forward's rows bit for bit) and bitwise preservation (a hash of the outputs on fixed seeded
+    inputs, compared with the hash recorded for the same contract id);
+  * verdict: verified / admissible / promoted against a recorded specification file.
+
+  python -m paper_2609_35140_b200.audit --record spec.json     # measure and write a baseline spec
+  python -m paper_2609_35140_b200.audit --check spec.json      # measure and judge against it
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import math
+from typing import Dict, List, Optional
+
+PREFILL_TOKENS = [1024, 4096, 8192, 16384]
+DECODE_CONTEXTS = [128, 1024, 4096, 8192]
+DECODE_BATCHES = [1, 4, 8, 16]
+HEADS = (32, 8, 128, 64)          # Hq, Hkv, head_dim, page size
+MAX_SLOWDOWN = 1.1                # per-workload limit relative to the recorded baseline
+
+
+def workload_names() -> List[str]:
+    names = ["prefill_%d_bs1" % n for n in PREFILL_TOKENS]
+    names += ["decode_ctx%d_bs%d" % (c, b) for c in DECODE_CONTEXTS for b in DECODE_BATCHES]
+    return names
+
+
+def aggregate(latencies_ms: Dict[str, float], weights: Optional[Dict[str, float]] = None) -> float:
+    """T = sum_w c_w * lat(w) with unit weights unless given (Eq. 2)."""
+    return float(sum((weights or {}).get(k, 1.0) * v for k, v in latencies_ms.items()))
+
+
+def judge(spec: dict, latencies_ms: Dict[str, float], checks_passed: bool, contract: str,
+          hashes: Optional[Dict[str, str]] = None) -> dict:
+    """Applies the promotion rule.  `spec` holds baseline latencies, the incumbent's aggregate,
+    the slowdown limit and (per contract id) the recorded output hashes."""
+    missing = [k for k in spec["baseline_ms"] if k not in latencies_ms or not math.isfinite(latencies_ms[k])]
+    preserved = None
+    recorded = spec.get("hashes", {}).get(contract)
+    if recorded is not None and hashes is not None:
+        preserved = all(recorded.get(k) == v for k, v in hashes.items())
+    verified = bool(checks_passed) and preserved is not False
+    limit = spec.get("max_slowdown", MAX_SLOWDOWN)
+    over = {k: latencies_ms[k] / spec["baseline_ms"][k] for k in spec["baseline_ms"]
+            if k in latencies_ms and latencies_ms[k] > limit * spec["baseline_ms"][k]}
+    admissible = verified and not missing and not over
+    T = aggregate({k: latencies_ms[k] for k in spec["baseline_ms"] if k in latencies_ms})
+    promoted = admissible and T < spec["incumbent_T_ms"]
+    return {"verified": verified, "bitwise_preserved": preserved, "admissible": admissible,
+            "promoted": promoted, "T_ms": T, "incumbent_T_ms": spec["incumbent_T_ms"],
+            "speedup_over_baseline": spec["baseline_T_ms"] / T if T > 0 else None,
+            "over_limit": over, "missing": missing}
+
+
+# ------------------------------------------------------------------------------------------ GPU part
+def _measure(fn, reps: int = 20, warmup: int = 3, flush=None) -> float:
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(reps):
+        if flush is not None:
+            flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    times.sort()
+    return float(times[len(times) // 2])
+
+
+def run_grid(reps: int = 20) -> Dict[str, float]:
+    """Median latency (ms, cold L2) of every workload of the grid."""
+    import numpy as np
+    import torch
+    from . import binding as tik
+    from . import synth
+    Hq, Hkv, d, page = HEADS
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    out: Dict[str, float] = {}
+    # one pool holds 16 sequences of 8192 tokens (decode) / one of 16384 (prefill)
+    w = synth.custom_workload([16384], [0], Hq, Hkv, d, page, index=70)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    layout = synth.make_paged_layout(w)
+    bt = torch.from_numpy(layout.block_table).cuda()
+    kc = torch.zeros(layout.num_pages, Hkv, page, d, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    tik.tik_kv_cache_write(k, v, cu, torch.tensor([16384], dtype=torch.int32, device="cuda"), kc, vc, bt)
+    for n in PREFILL_TOKENS:
+        cu_q = torch.tensor([0, n], dtype=torch.int32, device="cuda")
+        ctx = torch.tensor([n], dtype=torch.int32, device="cuda")
+        qn = q[:n].contiguous()
+        o = torch.empty_like(qn)
+        out["prefill_%d_bs1" % n] = _measure(
+            lambda: tik.tik_attn_prefill(qn, cu_q, ctx, kc, vc, bt, n, n, w.softmax_scale, o=o), reps, 3, flush)
+    wd = synth.custom_workload([8192] * 16, [0] * 16, Hq, Hkv, d, page, index=71)
+    q, k, v, cu = synth.make_qkv(wd, "cuda")
+    layout = synth.make_paged_layout(wd)
+    bt = torch.from_numpy(layout.block_table).cuda()
+    kc = torch.zeros(layout.num_pages, Hkv, page, d, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    tik.tik_kv_cache_write(k, v, cu, torch.tensor([8192] * 16, dtype=torch.int32, device="cuda"), kc, vc, bt)
+    cu_h = wd.cu_seqlens()
+    for c in DECODE_CONTEXTS:
+        for b in DECODE_BATCHES:
+            rows = torch.tensor([int(cu_h[s]) + c - 1 for s in range(b)], device="cuda")
+            qd = q[rows].contiguous()
+            ctx = torch.full((b,), c, dtype=torch.int32, device="cuda")
+            btb = bt[:b].contiguous()
+            o = torch.empty_like(qd)
+            ws = torch.empty(max(16, tik.workspace_bytes(tik.OP_ATTN_DECODE, b, Hq, Hkv, d, c)), dtype=torch.uint8,
+                             device="cuda")
+            out["decode_ctx%d_bs%d" % (c, b)] = _measure(
+                lambda: tik.tik_attn_decode(qd, ctx, kc, vc, btb, c, wd.softmax_scale, ws=ws, o=o), reps, 3, flush)
+    return out
+
+
+def run_checks() -> (bool, Dict[str, str]):
+    """Entry-point consistency on fixed seeded inputs plus the hashes of the outputs."""
+    import numpy as np
+    import torch
+    from . import binding as tik
+    from . import synth
+    ok = True
+    hashes: Dict[str, str] = {}
+    cases = {
+        "d128_g4": synth.custom_workload([300, 1024, 65], [200, 1100, 2000], 8, 2, 128, 64, index=80),
+        "d64_g4": synth.custom_workload([64, 64], [32, 96], 4, 1, 64, 16, index=81),
+    }
+    for name, w in cases.items():
+        q, k, v, cu = synth.make_qkv(w, "cuda")
+        o_train = tik.tik_attn_train_fwd(q, k, v, cu, max(w.seq_lens), w.softmax_scale)
+        layout = synth.make_paged_layout(w)
+        bt = torch.from_numpy(layout.block_table).cuda()
+        kc = torch.zeros(layout.num_pages, w.Hkv, layout.page_size, w.d, dtype=torch.bfloat16, device="cuda")
+        vc = torch.zeros_like(kc)
+        ctx = torch.tensor(w.seq_lens, dtype=torch.int32, device="cuda")
+        tik.tik_kv_cache_write(k, v, cu, ctx, kc, vc, bt)
+        o_pre = tik.tik_attn_prefill(q, cu, ctx, kc, vc, bt, max(w.seq_lens), max(w.seq_lens), w.softmax_scale)
+        ok &= bool(torch.equal(o_pre.view(torch.int16), o_train.view(torch.int16)))
+        cu_h = w.cu_seqlens()
+        for frac in (1.0, 0.6, 0.3):
+            pos = [max(1, int(L * frac)) - 1 for L in w.seq_lens]
+            rows = torch.tensor([int(cu_h[s]) + p for s, p in enumerate(pos)], device="cuda")
+            c2 = torch.tensor([p + 1 for p in pos], dtype=torch.int32, device="cuda")
+            o_dec = tik.tik_attn_decode(q[rows].contiguous(), c2, kc, vc, bt, max(pos) + 1, w.softmax_scale)
+            ok &= bool(torch.equal(o_dec.view(torch.int16), o_train[rows].view(torch.int16)))
+        hashes[name] = hashlib.sha256(o_train.view(torch.int16).cpu().numpy().tobytes()).hexdigest()
+    w = synth.get_workload(0)
+    hidden, W, target = synth.make_logprob_inputs(w, "cuda")
+    lp = tik.tik_token_logprob(hidden, W, target)
+    hashes["logprob_tiny"] = hashlib.sha256(lp.view(torch.int32).cpu().numpy().tobytes()).hexdigest()
+    ok &= tik.device_status() == 0
+    return ok, hashes
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
+    ap.add_argument("--record", metavar="SPEC", help="measure and write a baseline specification")
+    ap.add_argument("--check", metavar="SPEC", help="measure and judge against a specification")
+    ap.add_argument("--reps", type=int, default=20)
+    args = ap.parse_args()
+    from . import binding as tik
+    tik.load()
+    contract = tik.contract_id()
+    ok, hashes = run_checks()
+    lat = run_grid(args.reps)
+    if args.record:
+        T = aggregate(lat)
+        spec = {"hardware": "B200", "heads": HEADS, "weights": "unit", "max_slowdown": MAX_SLOWDOWN,
+                "baseline_ms": lat, "baseline_T_ms": T, "incumbent_T_ms": T,
+                "hashes": {contract: hashes}, "checks_passed": ok}
+        with open(args.record, "w") as f:
+            json.dump(spec, f, indent=1)
+        print(json.dumps({"recorded": args.record, "T_ms": T, "checks_passed": ok, "contract": contract}))
+    elif args.check:
+        with open(args.check) as f:
+            spec = json.load(f)
+        print(json.dumps({"contract": contract, "latencies_ms": lat, **judge(spec, lat, ok, contract, hashes)}))
+    else:
+        print(json.dumps({"contract": contract, "checks_passed": ok, "T_ms": aggregate(lat), "latencies_ms": lat,
+                          "hashes": hashes}))
+
+
+if __name__ == "__main__":
+    main()
