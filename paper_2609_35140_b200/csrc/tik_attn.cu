@@ -133,30 +133,107 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 268);
     float* lx = reinterpret_cast<float*>(smem + L::OFF_LX);
 
-    if (tid == 0) {
-        mbar_init(bar_q, 1);
-        for (int i = 0; i < KV_STAGES; ++i) {
-            mbar_init(bar_kfull + 8 * i, 1);
-            mbar_init(bar_vfull + 8 * i, 1);
-            mbar_init(bar_kempty + 8 * i, 1);
-            mbar_init(bar_vempty + 8 * i, 1);
+    // ---------------------------------------------------------------- set-up
+    // The two TMA warps initialise the barriers of their own rings and put the first K / V tiles
+    // (and Q) in flight before the CTA-wide synchronisation: a CTA's first data then arrives while
+    // TMEM is being allocated instead of ~1000 cycles later.
+    const int kv = (warp == 2) ? 1 : 0;                     // producer warps: 0 streams K, 2 streams V
+    const CUtensorMap* tm = kv ? &tmV : &tmK;
+    int my_phys = p.num_pages;                              // paged regimes: one block-table entry per lane
+    auto produce_tile = [&](int it) {                       // whole warp (paged) or lane 0 (train)
+        const int j = tile_first + it;
+        const int st = it % KV_STAGES;
+        const uint32_t use = it / KV_STAGES;
+        const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
+        const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
+        if (MODE != MODE_TRAIN) {
+            // Paged K/V: the warp reads 32 block-table entries at a time (one per lane, coalesced),
+            // so the table's latency is paid once per 32 pages instead of before every tile.
+            const int tiles_per_batch = 32 / p.pages_per_tile;
+            if (it % tiles_per_batch == 0) {
+                const int lp = (128 * j) / p.page_size + lane;
+                int ph = p.num_pages;       // out of range: the box is filled with zeros
+                if (lp * p.page_size < ctx) {
+                    ph = (lp < p.max_blocks) ? p.block_table[static_cast<long long>(seq) * p.max_blocks + lp] : -1;
+                    if (ph < 0 || ph >= p.num_pages) {
+                        if (kv == 0) atomicOr(p.dev_status, TIK_DEV_BAD_BLOCK);
+                        ph = p.num_pages;
+                    }
+                }
+                my_phys = ph;
+            }
         }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_sfull + 8 * i, 1);
-            mbar_init(bar_pfull + 8 * i, 4);
-            mbar_init(bar_sempty + 8 * i, 4);
-            mbar_init(bar_pempty + 8 * i, 1);
+        // Each stage has its own release barrier with this warp as its only waiter: a barrier
+        // shared with waiters of a different lag could run two phases ahead of the slowest one,
+        // which a parity wait cannot tell from "not yet".
+        if (use > 0)
+            mbar_wait((kv ? bar_vempty : bar_kempty) + 8 * st, (use - 1) & 1, abort_word, p.dev_status);
+        if (lane == 0) mbar_expect_tx(full, L::TILE);
+        if (MODE == MODE_TRAIN) {
+            if (lane == 0) {
+                const int row = static_cast<int>(tok0) + 128 * j;
+                for (int a = 0; a < NATOM; ++a) tma_load_3d(dst + a * L::ATOM, tm, full, a * 64, kvh, row);
+            }
+        } else {
+            const int ppt = p.pages_per_tile;
+            const int in_batch = it % (32 / ppt);
+            for (int i = 0; i < ppt; ++i) {
+                const int phys = __shfl_sync(0xffffffffu, my_phys, in_batch * ppt + i);
+                if (lane == 0) {
+                    const uint32_t off = static_cast<uint32_t>(i * p.page_size) * 128u;
+                    for (int a = 0; a < NATOM; ++a)
+                        tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, phys);
+                }
+            }
         }
-        for (int i = 0; i < 4; ++i) mbar_init(bar_hand + 8 * i, 1);
-        *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
-        fence_barrier_init();
-        tma_prefetch_desc(&tmQ);
-        tma_prefetch_desc(&tmK);
-        tma_prefetch_desc(&tmV);
-    }
-    if (warp == 1) {
+    };
+    auto load_q = [&]() {                                   // lane 0 of warp 0
+        if (MODE == MODE_DECODE) {
+            mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
+            for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
+        } else {
+            mbar_expect_tx(bar_q, L::TILE);
+            for (int a = 0; a < NATOM; ++a)
+                tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
+        }
+    };
+    const int n_early = min(n_tiles, KV_STAGES);            // tiles that need no stage release
+    if (warp == 0 || warp == 2) {
+        if (lane == 0) {
+            tma_prefetch_desc(tm);
+            if (kv == 0) {
+                tma_prefetch_desc(&tmQ);
+                mbar_init(bar_q, 1);
+            }
+            for (int i = 0; i < KV_STAGES; ++i) {
+                mbar_init((kv ? bar_vfull : bar_kfull) + 8 * i, 1);
+                mbar_init((kv ? bar_vempty : bar_kempty) + 8 * i, 1);
+            }
+            fence_barrier_init();
+            if (kv == 0 && MODE != MODE_DECODE) load_q();
+        }
+        __syncwarp();
+        if (MODE != MODE_TRAIN || lane == 0)
+            for (int it = 0; it < n_early; ++it) produce_tile(it);
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(bar_sfull + 8 * i, 1);
+                mbar_init(bar_pfull + 8 * i, 4);
+                mbar_init(bar_sempty + 8 * i, 4);
+                mbar_init(bar_pempty + 8 * i, 1);
+            }
+            for (int i = 0; i < 4; ++i) mbar_init(bar_hand + 8 * i, 1);
+            fence_barrier_init();
+        }
+        __syncwarp();
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
         tmem_relinquish();
+    } else if (warp == 3) {
+        // an earlier kernel on this context may have run out of a wait: then do nothing at all
+        if (lane == 0)
+            *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
     }
     if (MODE == MODE_DECODE) {
         // rows >= G of the Q tile are never loaded: zero them (their scores and weights stay 0)
@@ -180,73 +257,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // ------------------------------------------------------------ TMA producers
         // warp 0 streams Q and the K tiles, warp 2 the V tiles: a K tile is requested as soon as
         // the QK^T that used its stage has finished, without queueing behind a wait for PV.
-        const int kv = (warp == 2) ? 1 : 0;
-        const CUtensorMap* tm = kv ? &tmV : &tmK;
-        if (kv == 0 && lane == 0) {
-            if (MODE == MODE_DECODE) {
-                mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
-                for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
-            } else {
-                mbar_expect_tx(bar_q, L::TILE);
-                for (int a = 0; a < NATOM; ++a)
-                    tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
-            }
-        }
-        if (MODE == MODE_TRAIN) {
-            if (lane == 0) {
-                for (int it = 0; it < n_tiles; ++it) {
-                    if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
-                    const int st = it % KV_STAGES;
-                    const uint32_t use = it / KV_STAGES;
-                    const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
-                    const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
-                    // Each stage has its own release barrier with this thread as its only waiter: a
-                    // barrier shared with waiters of a different lag could run two phases ahead of
-                    // the slowest one, which a parity wait cannot tell from "not yet".
-                    if (use > 0)
-                        mbar_wait((kv ? bar_vempty : bar_kempty) + 8 * st, (use - 1) & 1, abort_word, p.dev_status);
-                    mbar_expect_tx(full, L::TILE);
-                    const int row = static_cast<int>(tok0) + 128 * (tile_first + it);
-                    for (int a = 0; a < NATOM; ++a) tma_load_3d(dst + a * L::ATOM, tm, full, a * 64, kvh, row);
-                }
-            }
-        } else {
-            // Paged K/V: the warp reads 32 block-table entries at a time (one per lane, coalesced),
-            // so the table's latency is paid once per 32 pages instead of before every tile.
-            const int ppt = p.pages_per_tile;
-            const int tiles_per_batch = 32 / ppt;
-            int my_phys = p.num_pages;
-            for (int it = 0; it < n_tiles; ++it) {
-                if (*abort_word) break;
-                const int j = tile_first + it;
-                const int in_batch = it % tiles_per_batch;
-                if (in_batch == 0) {
-                    const int lp = (128 * j) / p.page_size + lane;
-                    int ph = p.num_pages;       // out of range: the box is filled with zeros
-                    if (lp * p.page_size < ctx) {
-                        ph = (lp < p.max_blocks) ? p.block_table[static_cast<long long>(seq) * p.max_blocks + lp] : -1;
-                        if (ph < 0 || ph >= p.num_pages) {
-                            if (kv == 0) atomicOr(p.dev_status, TIK_DEV_BAD_BLOCK);
-                            ph = p.num_pages;
-                        }
-                    }
-                    my_phys = ph;
-                }
-                const int st = it % KV_STAGES;
-                const uint32_t use = it / KV_STAGES;
-                const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
-                const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
-                if (use > 0)
-                    mbar_wait((kv ? bar_vempty : bar_kempty) + 8 * st, (use - 1) & 1, abort_word, p.dev_status);
-                if (lane == 0) mbar_expect_tx(full, L::TILE);
-                for (int i = 0; i < ppt; ++i) {
-                    const int phys = __shfl_sync(0xffffffffu, my_phys, in_batch * ppt + i);
-                    if (lane == 0) {
-                        const uint32_t off = static_cast<uint32_t>(i * p.page_size) * 128u;
-                        for (int a = 0; a < NATOM; ++a)
-                            tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, phys);
-                    }
-                }
+        if (MODE == MODE_DECODE && kv == 0 && lane == 0) load_q();     // after the zero fill of the Q tile
+        if (MODE != MODE_TRAIN || lane == 0) {
+            for (int it = n_early; it < n_tiles; ++it) {
+                if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
+                produce_tile(it);
             }
         }
         __syncwarp();
