@@ -51,6 +51,12 @@ static tik_status cuda_fail(tik_ctx* ctx, cudaError_t e, const char* where) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static bool page_ok(int page) { return page == 16 || page == 32 || page == 64 || page == 128; }
 static float scale_to_c(float softmax_scale) { return softmax_scale * LOG2E_F; }
+// Candidate work items per (sequence, head) for the full-sequence kernels: query tiles 0..15 go
+// in pairs (x = 0..7), tiles >= 16 one by one (x = 8 + tile - 16); see attn_kernel.
+static unsigned attn_grid_x(int max_positions) {
+    const int nt = (max_positions + 127) / 128;
+    return static_cast<unsigned>(nt <= 16 ? (nt + 1) / 2 : 8 + (nt - 16));
+}
 
 static tik_status check_heads(tik_ctx* ctx, int Hq, int Hkv, int d, float scale) {
     if (Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return fail(ctx, TIK_ERR_INVALID_ARG, "Hq must be a positive multiple of Hkv");
@@ -171,6 +177,7 @@ tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const 
         return fail(ctx, TIK_ERR_CUDA, err.c_str());
 
     AttnParams p{};
+    if (!make_tmap_bf16(ctx, &p.tmO, o, 3, qd, qs, box, &err)) return fail(ctx, TIK_ERR_CUDA, err.c_str());
     p.o = o;
     p.lse = lse;
     p.cu_seqlens = cu_seqlens;
@@ -179,7 +186,7 @@ tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const 
     p.G = Hq / Hkv;
     p.c = scale_to_c(softmax_scale);
     p.dev_status = ctx->dev_status;
-    dim3 grid((max_seqlen + 127) / 128, Hq, S);
+    dim3 grid(attn_grid_x(max_seqlen), Hq, S);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
     cudaError_t e = launch_attn(d, 0, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_train_fwd");
@@ -248,6 +255,7 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
     if (s != TIK_OK) return s;
 
     AttnParams p{};
+    if (!make_tmap_bf16(ctx, &p.tmO, o, 3, qd, qs, box, &err)) return fail(ctx, TIK_ERR_CUDA, err.c_str());
     p.o = o;
     p.lse = lse;
     p.cu_seqlens = cu_seqlens_q;
@@ -262,8 +270,8 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
     p.num_pages = num_pages;
     p.c = scale_to_c(softmax_scale);
     p.dev_status = ctx->dev_status;
-    // query tiles are aligned to absolute positions: an unaligned start adds one tile
-    dim3 grid((max_q_len + 127) / 128 + 1, Hq, S);
+    // query tiles are aligned to absolute positions 0 .. ctx-1 (tiles before the first new token exit)
+    dim3 grid(attn_grid_x(max_ctx_len), Hq, S);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
     cudaError_t e = launch_attn(d, 1, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_prefill");

@@ -33,8 +33,10 @@ template <int D>
 struct AttnSmem {
     static constexpr uint32_t ATOM = 128 * 128;          // 128 rows x 64 bf16
     static constexpr uint32_t TILE = (D / 64) * ATOM;    // one Q, K or V tile
+    // seven tiles: one query tile + three K stages + three V stages, or (paired mode) two query
+    // tiles + two K stages + three V stages
     static constexpr uint32_t OFF_Q = 0;
-    static constexpr uint32_t OFF_K = TILE;
+    static constexpr uint32_t OFF_K = TILE;                        // paired mode: 2 * TILE
     static constexpr uint32_t OFF_V = OFF_K + KV_STAGES * TILE;
     static constexpr uint32_t OFF_BAR = OFF_V + KV_STAGES * TILE;
     static constexpr uint32_t OFF_LX = OFF_BAR + 272;             // 3 x 128 floats of row state
@@ -45,7 +47,7 @@ struct AttnSmem {
 template <int D, int MODE>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-            const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+            const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnParams p) {
     using L = AttnSmem<D>;
     constexpr int NATOM = D / 64;
     constexpr int DH = D / 2;                              // O columns owned by one softmax thread
@@ -59,41 +61,57 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---------------------------------------------------------------- work item
-    int seq, head, kvh, T = 0, chunk = 0, ctx = 0, pos0 = 0;
-    long long qrow0 = 0;       // token row of tile row 0 (train/prefill), may be negative
-    long long tok0 = 0;        // first token of the sequence in the packed K/V (train)
-    int row_lo = 0, row_hi = 0;   // valid tile rows [row_lo, row_hi)
+    // Train / prefill: query tiles are aligned to absolute positions.  Tiles 0..15 (their KV
+    // range is one chunk) are taken two at a time: a CTA owns tiles 2m (A) and 2m+1 (B) of one
+    // (sequence, head), streams every K/V tile once for both, and each softmax warpgroup keeps
+    // the rows of one of the two tiles from the first KV tile to the last.  Tiles >= 16, a tile
+    // without a partner, and decode run one query tile per CTA.
+    int seq, head, kvh, chunk = 0, ctx = 0;
+    int T0 = 0, T1 = 0;        // query tile of parity 0 (single mode, or B) and of parity 1 (A)
+    bool pair = false;
+    long long qrow0[2] = {0, 0};   // token row of tile row 0, per query tile (may be negative)
+    long long tok0 = 0;            // first token of the sequence in the packed K/V (train)
+    int row_lo[2] = {0, 0}, row_hi[2] = {0, 0};   // valid tile rows [row_lo, row_hi), per query tile
     int tile_first, tile_last;
-    if (MODE == MODE_TRAIN) {
+    if (MODE == MODE_TRAIN || MODE == MODE_PREFILL) {
         seq = blockIdx.z;
         head = blockIdx.y;
         kvh = head / p.G;
-        T = gridDim.x - 1 - blockIdx.x;
-        tok0 = p.cu_seqlens[seq];
-        const int len = p.cu_seqlens[seq + 1] - static_cast<int>(tok0);
-        if (128 * T >= len) return;
-        ctx = len;
-        qrow0 = tok0 + 128ll * T;
-        row_lo = 0;
-        row_hi = min(128, len - 128 * T);
+        int pos0, qb;
+        if (MODE == MODE_TRAIN) {
+            tok0 = p.cu_seqlens[seq];
+            ctx = p.cu_seqlens[seq + 1] - static_cast<int>(tok0);
+            pos0 = 0;
+            qb = static_cast<int>(tok0);
+            if (ctx <= 0) return;
+        } else {
+            qb = p.cu_seqlens[seq];
+            const int qlen = p.cu_seqlens[seq + 1] - qb;
+            ctx = p.ctx_lens[seq];
+            pos0 = ctx - qlen;
+            if (qlen <= 0 || pos0 < 0) return;
+        }
+        const int t_lo = pos0 / 128, t_hi = (ctx - 1) / 128;     // first and last query tile
+        const int x = gridDim.x - 1 - blockIdx.x;                // heaviest candidates first
+        if (x >= 8) {
+            T0 = 16 + (x - 8);
+            if (T0 < t_lo || T0 > t_hi) return;
+        } else {
+            const int ta = 2 * x, tb = 2 * x + 1;
+            const bool va = ta >= t_lo && ta <= t_hi, vb = tb >= t_lo && tb <= t_hi;
+            if (!va && !vb) return;
+            pair = va && vb;
+            T0 = vb ? tb : ta;
+            T1 = ta;
+        }
+        for (int q2 = 0; q2 < 2; ++q2) {
+            const int Tq = q2 ? T1 : T0;
+            qrow0[q2] = static_cast<long long>(qb) + 128ll * Tq - pos0;
+            row_lo[q2] = max(0, pos0 - 128 * Tq);
+            row_hi[q2] = min(128, ctx - 128 * Tq);
+        }
         tile_first = 0;
-        tile_last = T;
-    } else if (MODE == MODE_PREFILL) {
-        seq = blockIdx.z;
-        head = blockIdx.y;
-        kvh = head / p.G;
-        const int qb = p.cu_seqlens[seq];
-        const int qlen = p.cu_seqlens[seq + 1] - qb;
-        ctx = p.ctx_lens[seq];
-        pos0 = ctx - qlen;
-        if (qlen <= 0 || pos0 < 0) return;
-        T = pos0 / 128 + (gridDim.x - 1 - blockIdx.x);
-        if (128 * T >= ctx) return;
-        qrow0 = static_cast<long long>(qb) + 128ll * T - pos0;
-        row_lo = max(0, pos0 - 128 * T);
-        row_hi = min(128, ctx - 128 * T);
-        tile_first = 0;
-        tile_last = T;
+        tile_last = T0;
     } else {
         seq = blockIdx.z;
         kvh = blockIdx.y;
@@ -103,10 +121,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         if (ctx <= 0 || chunk * CHUNK >= ctx) return;
         tile_first = chunk * TILES_PER_CHUNK;
         tile_last = min(tile_first + TILES_PER_CHUNK - 1, (ctx - 1) / 128);
-        row_lo = 0;
-        row_hi = p.G;
+        row_lo[0] = 0;
+        row_hi[0] = p.G;
     }
-    const int n_tiles = tile_last - tile_first + 1;
+    const int n_tiles = tile_last - tile_first + 1;              // K/V tiles streamed by this CTA
+    // One step = one (query tile, KV tile) product.  Single mode: step g is KV tile g.  Paired
+    // mode: even steps belong to B (= T0), odd steps to A (= T1 = T0 - 1), step g uses KV tile g/2;
+    // A has one KV tile less, so the last step (even) is B's diagonal tile.
+    const int n_steps = pair ? (2 * n_tiles - 1) : n_tiles;
+    const int KS = pair ? 2 : KV_STAGES;                         // K stages in use
+    const int q_row_first[2] = {static_cast<int>(qrow0[0]), static_cast<int>(qrow0[1])};
 
     // ---------------------------------------------------------------- shared memory
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -116,7 +140,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         if (tid == 0) atomicOr(p.dev_status, TIK_DEV_WAIT_EXPIRED);
         return;
     }
-    const uint32_t sQ = sbase + L::OFF_Q, sK = sbase + L::OFF_K, sV = sbase + L::OFF_V;
+    const uint32_t sQ = sbase + L::OFF_Q, sK = sbase + (pair ? 2 * L::TILE : L::OFF_K), sV = sbase + L::OFF_V;
     // barriers (8 bytes each)
     const uint32_t bar0 = sbase + L::OFF_BAR;
     const uint32_t bar_q = bar0;                 // Q landed
@@ -132,6 +156,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 264);
     volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 268);
     float* lx = reinterpret_cast<float*>(smem + L::OFF_LX);
+    // values only the epilogue needs are parked in shared memory instead of living in registers
+    // across the main loop: [q2][0] first token row, [q2][1] row_lo, [q2][2] row_hi
+    volatile int* meta = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 216);
+    if (tid == 64) {
+        for (int q2 = 0; q2 < 2; ++q2) {
+            meta[3 * q2] = q_row_first[q2];
+            meta[3 * q2 + 1] = row_lo[q2];
+            meta[3 * q2 + 2] = row_hi[q2];
+        }
+    }
 
     // ---------------------------------------------------------------- set-up
     // The two TMA warps initialise the barriers of their own rings and put the first K / V tiles
@@ -142,8 +176,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     int my_phys = p.num_pages;                              // paged regimes: one block-table entry per lane
     auto produce_tile = [&](int it) {                       // whole warp (paged) or lane 0 (train)
         const int j = tile_first + it;
-        const int st = it % KV_STAGES;
-        const uint32_t use = it / KV_STAGES;
+        const int nst = kv ? KV_STAGES : KS;
+        const int st = it % nst;
+        const uint32_t use = it / nst;
         const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
         const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
         if (MODE != MODE_TRAIN) {
@@ -192,12 +227,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
             for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
         } else {
-            mbar_expect_tx(bar_q, L::TILE);
-            for (int a = 0; a < NATOM; ++a)
-                tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, static_cast<int>(qrow0));
+            mbar_expect_tx(bar_q, pair ? 2 * L::TILE : L::TILE);
+            for (int q2 = 0; q2 < (pair ? 2 : 1); ++q2)
+                for (int a = 0; a < NATOM; ++a)
+                    tma_load_3d(sQ + q2 * L::TILE + a * L::ATOM, &tmQ, bar_q, a * 64, head,
+                                static_cast<int>(qrow0[q2]));
         }
     };
-    const int n_early = min(n_tiles, KV_STAGES);            // tiles that need no stage release
+    const int n_early = min(n_tiles, kv ? KV_STAGES : KS);  // tiles that need no stage release
     if (warp == 0 || warp == 2) {
         if (lane == 0) {
             tma_prefetch_desc(tm);
@@ -269,38 +306,45 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // ------------------------------------------------------------ QK^T issuer
         // Two threads feed the tensor pipe (this one and the PV issuer in warp 3): whatever an
         // issuing thread executes between MMAs is time in which it queues nothing, so each
-        // keeps to waits, one MMA chain and one commit per tile.
+        // keeps to waits, one MMA chain and its commits per step.
         if (lane == 0) {
             mbar_wait(bar_q, 0, abort_word, p.dev_status);
-            const uint64_t dq = smem_desc_sw128(sQ, 0, 1024);
-            for (int x = 0; x < n_tiles; ++x) {
-                const int st = x % KV_STAGES, b = x & 1;
-                // the single score buffer is free once the softmax of tile x-1 holds it in registers
-                if (x >= 1) mbar_wait(bar_sempty + 8 * ((x - 1) & 1), ((x - 1) >> 1) & 1, abort_word, p.dev_status);
-                mbar_wait(bar_kfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
+            const uint64_t dq0 = smem_desc_sw128(sQ, 0, 1024);
+            const uint64_t dq1 = smem_desc_sw128(sQ + L::TILE, 0, 1024);
+            for (int g = 0; g < n_steps; ++g) {
+                const int kt = pair ? (g >> 1) : g;                 // K tile of this step
+                const int st = kt % KS, b = g & 1;
+                // the single score buffer is free once the softmax of step g-1 holds it in registers
+                if (g >= 1) mbar_wait(bar_sempty + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_word, p.dev_status);
+                mbar_wait(bar_kfull + 8 * st, (kt / KS) & 1, abort_word, p.dev_status);
                 tc_fence_after();
+                const uint64_t dq = (pair && b) ? dq1 : dq0;
                 const uint64_t dk = smem_desc_sw128(sK + st * L::TILE, 0, 1024);
                 if (D == 128) mma_ss_chain8_fresh(tmem + COL_S, dq, dk, IDESC_QK);
                 else mma_ss_chain4_fresh(tmem + COL_S, dq, dk, IDESC_QK);
                 mma_commit(bar_sfull + 8 * b);
-                mma_commit(bar_kempty + 8 * st);
+                // the K stage is free after its last reader (paired mode: the odd step, or B's last tile)
+                if (!pair || b || g == n_steps - 1) mma_commit(bar_kempty + 8 * st);
             }
         }
         __syncwarp();
     } else if (warp == 3) {
         // ------------------------------------------------------------ PV issuer
         if (lane == 0) {
-            for (int x = 0; x < n_tiles; ++x) {
-                const int st = x % KV_STAGES, b = x & 1;
-                mbar_wait(bar_vfull + 8 * st, (x / KV_STAGES) & 1, abort_word, p.dev_status);
-                mbar_wait(bar_pfull + 8 * b, (x >> 1) & 1, abort_word, p.dev_status);
+            for (int g = 0; g < n_steps; ++g) {
+                const int vt = pair ? (g >> 1) : g;
+                const int st = vt % KV_STAGES, b = g & 1;
+                mbar_wait(bar_vfull + 8 * st, (vt / KV_STAGES) & 1, abort_word, p.dev_status);
+                mbar_wait(bar_pfull + 8 * b, (g >> 1) & 1, abort_word, p.dev_status);
                 tc_fence_after();
+                // paired mode: B accumulates in O_A, A in O_B, each from its first KV tile on
+                const uint32_t col_o = pair ? (b ? COL_OB : COL_OA) : col_o_of(g);
+                const bool fresh = pair ? (vt == 0) : is_chunk_start(g);
                 // A = bf16 weights in TMEM (8 columns per 16 keys), B = V tile
-                mma_ts_chain8(tmem + col_o_of(x), tmem + COL_P + 64 * b,
-                              smem_desc_sw128(sV + st * L::TILE, L::ATOM, 1024), IDESC_PV,
-                              is_chunk_start(x) ? 0u : 1u);
+                mma_ts_chain8(tmem + col_o, tmem + COL_P + 64 * b,
+                              smem_desc_sw128(sV + st * L::TILE, L::ATOM, 1024), IDESC_PV, fresh ? 0u : 1u);
                 mma_commit(bar_pempty + 8 * b);
-                mma_commit(bar_vempty + 8 * st);
+                if (!pair || b || g == n_steps - 1) mma_commit(bar_vempty + 8 * st);
             }
         }
         __syncwarp();
@@ -317,7 +361,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         const int quarter = warp & 3;                       // TMEM lane quarter of this warp
         const int r = quarter * 32 + lane;                  // tile row == TMEM lane
         const uint32_t tlane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
-        const int qpos = (MODE == MODE_DECODE) ? (ctx - 1) : (128 * T + r);
+        const int qpos = (MODE == MODE_DECODE) ? (ctx - 1) : (128 * T0 + r);
         const bool active = (MODE != MODE_DECODE) || (quarter == 0);
         const float c = p.c;
         float* st_m = lx;                 // [128]    running maximum of the current chunk
@@ -370,6 +414,125 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         };
         const int last = n_tiles - 1;
 
+        if (pair) {
+            // ---- paired mode: this warpgroup keeps the rows of one query tile (wg 0: tile B = T0,
+            // wg 1: tile A = T1) through all of that tile's KV tiles; nothing is handed over.
+            const int Tq = wg ? T1 : T0;
+            const int qpos_p = 128 * Tq + r;
+            const uint32_t to = tlane + (wg ? COL_OB : COL_OA);
+            float m_run = -CUDART_INF_F, l_lo = 0.0f, l_hi = 0.0f;
+            int g_last = wg;
+            for (int g = wg; g < n_steps; g += 2) {
+                g_last = g;
+                const int j = g >> 1;
+                mbar_wait(bar_sfull + 8 * wg, (g >> 1) & 1, abort_word, p.dev_status);
+                // the PV of step g-2 read this warpgroup's weight buffer and updated its accumulator
+                if (g >= 2) wait_pv(g - 2);
+                tc_fence_after();
+                const int kmax = qpos_p - 128 * j;              // columns > kmax are masked
+                uint32_t sc[128];
+                tmem_ld32(ts, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+                tmem_ld32(ts + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[32]));
+                tmem_ld32(ts + 64, *reinterpret_cast<uint32_t(*)[32]>(&sc[64]));
+                tmem_ld32(ts + 96, *reinterpret_cast<uint32_t(*)[32]>(&sc[96]));
+                tmem_wait_ld();
+                // the scores are in registers: the next QK^T may overwrite the buffer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_sempty + 8 * wg);
+                if (kmax < 127) {
+#pragma unroll
+                    for (int i = 0; i < 128; ++i)
+                        if (i > kmax) sc[i] = 0xff800000u;          // -inf
+                }
+                float mx[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) mx[k] = fmaxf(__uint_as_float(sc[2 * k]), __uint_as_float(sc[2 * k + 1]));
+#pragma unroll
+                for (int i = 16; i < 128; i += 16) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        mx[k] = fmax3(mx[k], __uint_as_float(sc[i + 2 * k]), __uint_as_float(sc[i + 2 * k + 1]));
+                }
+                const float mt = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmax3(fmax3(mx[3], mx[4], mx[5]), mx[6], mx[7]));
+                const float m_new = softmax_next_max(m_run, mt, c);
+                const float neg_mc = -__fmul_rn(m_new, c);
+                const float alpha = softmax_alpha(m_run, m_new, c);
+                m_run = m_new;
+                RowSum4 rs_lo, rs_hi;
+                rs_lo.reset();
+                rs_hi.reset();
+#pragma unroll
+                for (int i = 0; i < 64; i += 8) softmax_p8(&sc[i], c, neg_mc, rs_lo, &sc[i >> 1]);
+                tmem_st32(tp, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+#pragma unroll
+                for (int i = 0; i < 64; i += 8) softmax_p8(&sc[64 + i], c, neg_mc, rs_hi, &sc[32 + (i >> 1)]);
+                tmem_st32(tp + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[32]));
+                l_lo = __fmaf_rn(l_lo, alpha, rs_lo.total());
+                l_hi = __fmaf_rn(l_hi, alpha, rs_hi.total());
+                if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.0f)) {
+                    // rescale this tile's accumulator (its last PV, step g-2, is complete)
+#pragma unroll
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        uint32_t v[32];
+                        tmem_ld32(to + 32 * cc, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
+                        tmem_st32(to + 32 * cc, v);
+                    }
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_pfull + 8 * wg);
+            }
+            // ---- this tile is complete after its last PV: normalise and store its rows
+            wait_pv(g_last);
+            const float Ltot = finalize_l(l_lo, l_hi);
+            const float inv = finalize_inv(Ltot);
+            const int e_row0 = meta[3 * wg], e_lo = meta[3 * wg + 1], e_hi = meta[3 * wg + 2];
+            const bool valid = (r >= e_lo) && (r < e_hi);
+            const long long orow = (static_cast<long long>(e_row0) + r) * p.Hq + head;
+            if (valid && p.lse) p.lse[orow] = finalize_lse(m_run, Ltot, c);
+            __nv_bfloat16* optr = reinterpret_cast<__nv_bfloat16*>(p.o) + orow * D;
+            // A complete tile leaves through shared memory (the tile's own, now idle, query
+            // buffer) and one tiled TMA store; a ragged tile is written row by row.
+            const bool full_tile = e_lo == 0 && e_hi == 128;
+            uint8_t* stage = smem + L::OFF_Q + wg * L::TILE;
+#pragma unroll
+            for (int cc = 0; cc < D / 32; ++cc) {
+                uint32_t v[32];
+                tmem_ld32(to + 32 * cc, v);
+                tmem_wait_ld();
+                uint32_t o16[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    o16[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv),
+                                         finalize_o(__uint_as_float(v[2 * i + 1]), inv));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 val = make_uint4(o16[4 * i], o16[4 * i + 1], o16[4 * i + 2], o16[4 * i + 3]);
+                    if (full_tile) {
+                        const int c16 = 4 * cc + i;             // 16-byte chunk of the row
+                        *reinterpret_cast<uint4*>(stage + (c16 >> 3) * L::ATOM + r * 128 + (((c16 & 7) ^ (r & 7)) << 4)) = val;
+                    } else if (valid) {
+                        reinterpret_cast<uint4*>(optr + 32 * cc)[i] = val;
+                    }
+                }
+            }
+            if (full_tile) {
+                fence_proxy_async_smem();
+                named_bar_sync(2 + wg, 128);
+                if (quarter == 0 && lane == 0) {
+                    for (int a = 0; a < NATOM; ++a)
+                        tma_store_3d(&p.tmO, smem_u32(stage) + a * L::ATOM, a * 64, head, e_row0);
+                    tma_store_commit();
+                    tma_store_wait_read();
+                }
+            }
+        } else {
         for (int it = wg; it < n_tiles; it += 2) {
             const int j = tile_first + it;
             const bool chunk_start = is_chunk_start(it);
@@ -496,8 +659,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     fold_chunk(chunk_of(last), m_own, l_own_lo, l_own_hi, true);
                     const float Ltot = finalize_l(Lg_lo, Lg_hi);
                     st_m[r] = finalize_inv(Ltot);       // the hand-off slots are free now
-                    const bool valid = (r >= row_lo) && (r < row_hi);
-                    if (valid && p.lse) p.lse[(qrow0 + r) * p.Hq + head] = finalize_lse(M_g, Ltot, c);
+                    const bool valid = (r >= meta[1]) && (r < meta[2]);
+                    if (valid && p.lse) p.lse[(static_cast<long long>(meta[0]) + r) * p.Hq + head] = finalize_lse(M_g, Ltot, c);
                 }
             }
             tc_fence_before();
@@ -524,27 +687,46 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
             } else {
                 const float inv = st_m[r];
-                const bool valid = (r >= row_lo) && (r < row_hi);
-                const long long orow = (qrow0 + r) * p.Hq + head;
+                const int e_row0 = meta[0], e_lo = meta[1], e_hi = meta[2];
+                const bool valid = (r >= e_lo) && (r < e_hi);
+                const long long orow = (static_cast<long long>(e_row0) + r) * p.Hq + head;
                 __nv_bfloat16* optr = reinterpret_cast<__nv_bfloat16*>(p.o) + orow * D + DH * wg;
+                const bool full_tile = e_lo == 0 && e_hi == 128;
+                uint8_t* stage = smem + L::OFF_Q;            // the query tile is no longer needed
 #pragma unroll
                 for (int cc = 0; cc < DH / 32; ++cc) {
                     uint32_t v[32];
                     tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, v);
                     tmem_wait_ld();
-                    if (valid) {
-                        uint32_t o16[16];
+                    uint32_t o16[16];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            o16[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv),
-                                                 finalize_o(__uint_as_float(v[2 * i + 1]), inv));
-                        uint4* dst = reinterpret_cast<uint4*>(optr + 32 * cc);
+                    for (int i = 0; i < 16; ++i)
+                        o16[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv),
+                                             finalize_o(__uint_as_float(v[2 * i + 1]), inv));
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            dst[i] = make_uint4(o16[4 * i], o16[4 * i + 1], o16[4 * i + 2], o16[4 * i + 3]);
+                    for (int i = 0; i < 4; ++i) {
+                        const uint4 val = make_uint4(o16[4 * i], o16[4 * i + 1], o16[4 * i + 2], o16[4 * i + 3]);
+                        if (full_tile) {
+                            const int c16 = (DH * wg) / 8 + 4 * cc + i;     // 16-byte chunk of the row
+                            *reinterpret_cast<uint4*>(stage + (c16 >> 3) * L::ATOM + r * 128 + (((c16 & 7) ^ (r & 7)) << 4)) = val;
+                        } else if (valid) {
+                            reinterpret_cast<uint4*>(optr + 32 * cc)[i] = val;
+                        }
+                    }
+                }
+                if (full_tile) {
+                    // a complete tile leaves through shared memory and one tiled TMA store
+                    fence_proxy_async_smem();
+                    named_bar_sync(1, 256);
+                    if (warp == 4 && lane == 0) {
+                        for (int a = 0; a < NATOM; ++a)
+                            tma_store_3d(&p.tmO, smem_u32(stage) + a * L::ATOM, a * 64, head, e_row0);
+                        tma_store_commit();
+                        tma_store_wait_read();
                     }
                 }
             }
+        }
         }
     }
 
