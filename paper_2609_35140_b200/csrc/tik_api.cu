@@ -186,6 +186,7 @@ tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const 
     p.G = Hq / Hkv;
     p.c = scale_to_c(softmax_scale);
     p.dev_status = ctx->dev_status;
+    p.lookahead = ctx->sm_count;
     dim3 grid(attn_grid_x(max_seqlen), Hq, S);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
     cudaError_t e = launch_attn(d, 0, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
@@ -270,6 +271,7 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
     p.num_pages = num_pages;
     p.c = scale_to_c(softmax_scale);
     p.dev_status = ctx->dev_status;
+    p.lookahead = ctx->sm_count;
     // query tiles are aligned to absolute positions 0 .. ctx-1 (tiles before the first new token exit)
     dim3 grid(attn_grid_x(max_ctx_len), Hq, S);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");

@@ -271,6 +271,38 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // an earlier kernel on this context may have run out of a wait: then do nothing at all
         if (lane == 0)
             *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
+        // Query tiles are read once, so a CTA's first load is a DRAM miss of ~1.5 us with nothing
+        // to overlap it.  CTAs start roughly in block order as SMs free up: prefetch into L2 the
+        // query tiles of the CTA that comes `lookahead` blocks later, which starts about when this
+        // one ends.
+        if (MODE != MODE_DECODE && lane == 0) {
+            const long long nblk = static_cast<long long>(gridDim.x) * gridDim.y * gridDim.z;
+            const long long lin = (static_cast<long long>(blockIdx.z) * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+            const long long nxt = lin + p.lookahead;
+            if (nxt < nblk) {
+                const int bx = static_cast<int>(nxt % gridDim.x);
+                const int by = static_cast<int>((nxt / gridDim.x) % gridDim.y);
+                const int bz = static_cast<int>(nxt / (static_cast<long long>(gridDim.x) * gridDim.y));
+                int qb2 = p.cu_seqlens[bz], ctx2, pos2;
+                if (MODE == MODE_TRAIN) {
+                    ctx2 = p.cu_seqlens[bz + 1] - qb2;
+                    pos2 = 0;
+                } else {
+                    ctx2 = p.ctx_lens[bz];
+                    pos2 = ctx2 - (p.cu_seqlens[bz + 1] - qb2);
+                }
+                if (ctx2 > 0 && pos2 >= 0) {
+                    const int x2 = gridDim.x - 1 - bx;
+                    const int t_lo2 = pos2 / 128, t_hi2 = (ctx2 - 1) / 128;
+                    for (int q2 = 0; q2 < 2; ++q2) {
+                        const int Tq = (x2 >= 8) ? (16 + x2 - 8) : (2 * x2 + q2);
+                        if ((x2 >= 8 && q2 == 1) || Tq < t_lo2 || Tq > t_hi2) continue;
+                        const int row = qb2 + 128 * Tq - pos2;
+                        for (int a = 0; a < NATOM; ++a) tma_prefetch_l2_3d(&tmQ, a * 64, by, row);
+                    }
+                }
+            }
+        }
     }
     if (MODE == MODE_DECODE) {
         // rows >= G of the Q tile are never loaded: zero them (their scores and weights stay 0)

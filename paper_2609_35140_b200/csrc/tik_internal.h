@@ -37,6 +37,7 @@ struct AttnParams {
     float* part_ml;              // decode: [B][Hq][nchunk_max][4] = m, l_lo, l_hi, unused
     int nchunk_max;
     int* dev_status;
+    int lookahead;               // train / prefill: block distance of the query-tile L2 prefetch
 };
 
 // mode: 0 train (packed K/V), 1 prefill (paged K/V), 2 decode (paged K/V, chunk partials)
