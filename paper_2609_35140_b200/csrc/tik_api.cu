@@ -325,7 +325,9 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     p.part_o = static_cast<float*>(ws);
     p.part_ml = p.part_o + static_cast<size_t>(B) * Hq * nchunk * d;
     p.dev_status = ctx->dev_status;
-    dim3 grid(nchunk, Hkv, B);
+    p.cpc = decode_chunks_per_cta(B, Hkv, nchunk, ctx->sm_count);
+    p.lookahead = ctx->sm_count;
+    dim3 grid((nchunk + p.cpc - 1) / p.cpc, Hkv, B);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hkv and B must be <= 65535");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = launch_attn(d, 2, grid, tmQ, tmK, tmV, p, st);

@@ -40,7 +40,11 @@ struct AttnSmem {
     static constexpr uint32_t OFF_V = OFF_K + KV_STAGES * TILE;
     static constexpr uint32_t OFF_BAR = OFF_V + KV_STAGES * TILE;
     static constexpr uint32_t OFF_LX = OFF_BAR + 272;             // 3 x 128 floats of row state
-    static constexpr uint32_t BYTES = OFF_LX + 3 * 512;
+    // decode: exchange area of the softmax warps (per warpgroup 3 x 8 x 32 float4 of weights and
+    // 4 x 32 tile maxima).  Decode uses two K stages, so for D = 128 the third K stage holds it.
+    static constexpr uint32_t XCH_WG = 3 * 8 * 32 * 16 + 4 * 32 * 4;
+    static constexpr uint32_t OFF_XCH = (2 * XCH_WG <= TILE) ? OFF_K + 2 * TILE : OFF_LX + 3 * 512;
+    static constexpr uint32_t BYTES = OFF_LX + 3 * 512 + ((2 * XCH_WG <= TILE) ? 0 : 2 * XCH_WG);
     static constexpr uint32_t ALLOC = BYTES;                      // base must be 1 KiB aligned
 };
 
@@ -116,11 +120,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         seq = blockIdx.z;
         kvh = blockIdx.y;
         head = kvh * p.G;
-        chunk = blockIdx.x;
+        // a CTA streams `cpc` consecutive chunks; each still leaves its own partial
+        chunk = blockIdx.x * p.cpc;
         ctx = p.ctx_lens[seq];
         if (ctx <= 0 || chunk * CHUNK >= ctx) return;
         tile_first = chunk * TILES_PER_CHUNK;
-        tile_last = min(tile_first + TILES_PER_CHUNK - 1, (ctx - 1) / 128);
+        tile_last = min(tile_first + p.cpc * TILES_PER_CHUNK - 1, (ctx - 1) / 128);
         row_lo[0] = 0;
         row_hi[0] = p.G;
     }
@@ -129,7 +134,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     // mode: even steps belong to B (= T0), odd steps to A (= T1 = T0 - 1), step g uses KV tile g/2;
     // A has one KV tile less, so the last step (even) is B's diagonal tile.
     const int n_steps = pair ? (2 * n_tiles - 1) : n_tiles;
-    const int KS = pair ? 2 : KV_STAGES;                         // K stages in use
+    const int KS = (pair || MODE == MODE_DECODE) ? 2 : KV_STAGES;   // K stages in use
     const int q_row_first[2] = {static_cast<int>(qrow0[0]), static_cast<int>(qrow0[1])};
 
     // ---------------------------------------------------------------- shared memory
@@ -224,8 +229,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     };
     auto load_q = [&]() {                                   // lane 0 of warp 0
         if (MODE == MODE_DECODE) {
-            mbar_expect_tx(bar_q, static_cast<uint32_t>(p.G) * 128u * NATOM);
-            for (int a = 0; a < NATOM; ++a) tma_load_3d(sQ + a * L::ATOM, &tmQ, bar_q, a * 64, head, seq);
+            // the G query rows go to rows 0.., 32.., 64.., 96..: every lane quarter of the score
+            // tile then holds the same G rows and the four warps of a warpgroup share a row's columns
+            mbar_expect_tx(bar_q, 4u * static_cast<uint32_t>(p.G) * 128u * NATOM);
+            for (int q4 = 0; q4 < 4; ++q4)
+                for (int a = 0; a < NATOM; ++a)
+                    tma_load_3d(sQ + a * L::ATOM + q4 * 4096, &tmQ, bar_q, a * 64, head, seq);
         } else {
             mbar_expect_tx(bar_q, pair ? 2 * L::TILE : L::TILE);
             for (int q2 = 0; q2 < (pair ? 2 : 1); ++q2)
@@ -319,7 +328,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     auto chunk_of = [&](int it) { return (tile_first + it) / TILES_PER_CHUNK; };
     auto is_chunk_start = [&](int it) { return ((tile_first + it) % TILES_PER_CHUNK) == 0; };
     auto col_o_of = [&](int it) -> uint32_t {
-        return (MODE == MODE_DECODE || chunk_of(it) == 0) ? COL_OA : COL_OB;
+        // train / prefill: chunk 0 accumulates in O_A (the folded accumulator), later chunks in O_B;
+        // decode: consecutive chunks alternate, each is written out as a partial of its own
+        if (MODE == MODE_DECODE) return (chunk_of(it) & 1) ? COL_OB : COL_OA;
+        return chunk_of(it) == 0 ? COL_OA : COL_OB;
     };
 
     if (warp == 0 || warp == 2) {
@@ -331,6 +343,27 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             for (int it = n_early; it < n_tiles; ++it) {
                 if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
                 produce_tile(it);
+            }
+        }
+        if (MODE == MODE_DECODE && !*abort_word) {
+            // This warp has requested its last tile; the SM asks nothing of HBM while the CTA
+            // drains and its successor sets up.  Fill that gap: pull into L2 the first K (V)
+            // tiles of the CTA `lookahead` blocks later, which starts about when this one ends.
+            const long long nblk = static_cast<long long>(gridDim.x) * gridDim.y * gridDim.z;
+            const long long lin = (static_cast<long long>(blockIdx.z) * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+            const long long nxt = lin + p.lookahead;
+            if (p.lookahead > 0 && nxt < nblk) {
+                const int bx = static_cast<int>(nxt % gridDim.x);
+                const int by = static_cast<int>((nxt / gridDim.x) % gridDim.y);
+                const int bz = static_cast<int>(nxt / (static_cast<long long>(gridDim.x) * gridDim.y));
+                const int ctx2 = p.ctx_lens[bz];
+                const int pos2 = bx * p.cpc * CHUNK;                 // first key position of that CTA
+                const int lp = pos2 / p.page_size + lane;
+                if (lane < KV_STAGES * p.pages_per_tile && lp < p.max_blocks && lp * p.page_size < ctx2) {
+                    const int ph = p.block_table[static_cast<long long>(bz) * p.max_blocks + lp];
+                    if (ph >= 0 && ph < p.num_pages)
+                        for (int a = 0; a < NATOM; ++a) tma_prefetch_l2_4d(tm, a * 64, 0, by, ph);
+                }
             }
         }
         __syncwarp();
@@ -444,9 +477,172 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
             }
         };
+        // decode: the partial of a finished chunk; the accumulator columns [col0, col0 + ncol)
+        auto write_partial_ml = [&](int chunk_idx, float m_c, float l_c_lo, float l_c_hi) {
+            if (r < p.G) {
+                const long long slot = (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk_idx;
+                p.part_ml[4 * slot] = m_c;
+                p.part_ml[4 * slot + 1] = l_c_lo;
+                p.part_ml[4 * slot + 2] = l_c_hi;
+            }
+        };
+        auto write_partial_o = [&](int chunk_idx, int col0, int ncol) {
+            const uint32_t to = tlane + ((chunk_idx & 1) ? COL_OB : COL_OA);
+            for (int cc = 0; cc < ncol / 32; ++cc) {
+                uint32_t v[32];
+                tmem_ld32(to + col0 + 32 * cc, v);
+                tmem_wait_ld();
+                if (r < p.G) {
+                    const long long slot =
+                        (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk_idx;
+                    float4* dst = reinterpret_cast<float4*>(p.part_o + slot * D + col0 + 32 * cc);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                             __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                }
+            }
+        };
         const int last = n_tiles - 1;
 
-        if (pair) {
+        if (MODE == MODE_DECODE) {
+            // ---- decode: only G rows are real, and one warp per row block would leave the exp2
+            // work of a tile on a single scheduler.  The query rows are replicated into every
+            // lane quarter instead, and warp `quarter` takes columns [32 quarter, 32 quarter + 32)
+            // of every row: tile maximum and reference maximum by an exchange through shared
+            // memory, exponentials on all four warps, and then warp 0 alone sums the 128 weights
+            // of a row in the contract's order, packs them and writes them to TMEM, so the
+            // numbers are those of the one-thread-per-row path.
+            float4* xs = reinterpret_cast<float4*>(smem + L::OFF_XCH + wg * L::XCH_WG);   // [3][8][32]
+            float* xm = reinterpret_cast<float*>(smem + L::OFF_XCH + wg * L::XCH_WG + 3 * 8 * 32 * 16);   // [4][32]
+            const uint32_t bar_m0 = bar_hand;
+            for (int it = wg; it < n_tiles; it += 2) {
+                const int j = tile_first + it;
+                const bool chunk_start = is_chunk_start(it);
+                const bool fold_now = chunk_start && it > 0;      // a finished chunk precedes this tile
+                mbar_wait(bar_sfull + 8 * wg, (it >> 1) & 1, abort_word, p.dev_status);
+                if (it >= 2) wait_pv(it - 2);
+                tc_fence_after();
+                uint32_t sc[32];
+                tmem_ld32(ts + 32 * quarter, sc);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_sempty + 8 * wg);
+                const int kmax = (ctx - 1) - 128 * j - 32 * quarter;    // own columns > kmax are masked
+                if (kmax < 31) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i > kmax) sc[i] = 0xff800000u;              // -inf
+                }
+                float mx[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) mx[k] = fmaxf(__uint_as_float(sc[2 * k]), __uint_as_float(sc[2 * k + 1]));
+#pragma unroll
+                for (int i = 8; i < 32; i += 8) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mx[k] = fmax3(mx[k], __uint_as_float(sc[i + 2 * k]), __uint_as_float(sc[i + 2 * k + 1]));
+                }
+                xm[quarter * 32 + lane] = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                // state handed over by the warpgroup that processed tile it-1
+                float m_old = -CUDART_INF_F, l_old_lo = 0.0f, l_old_hi = 0.0f;
+                float m_prev = 0.0f, l_prev_lo = 0.0f, l_prev_hi = 0.0f;   // finished chunk, if any
+                if (it > 0) {
+                    mbar_wait(bar_m0, (it - 1) & 1, abort_word, p.dev_status);
+                    if (!chunk_start) {
+                        m_old = st_m[lane];
+                    } else if (quarter == 0) {
+                        wait_tile_done(it - 1);
+                        m_prev = st_m[lane];
+                        l_prev_lo = st_l[lane];
+                        l_prev_hi = st_l[128 + lane];
+                    }
+                }
+                named_bar_sync(2 + wg, 128);                 // maxima exchanged, old reference read by all
+                const float mt = fmaxf(fmaxf(xm[lane], xm[32 + lane]), fmaxf(xm[64 + lane], xm[96 + lane]));
+                const float m_new = softmax_next_max(m_old, mt, c);
+                if (quarter == 0) {
+                    st_m[lane] = m_new;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_m0);
+                }
+                const float neg_mc = -__fmul_rn(m_new, c);
+                float x[128];                                // warps 1-3 use the first 32 only
+#pragma unroll
+                for (int i = 0; i < 32; i += 8) softmax_x8(&sc[i], c, neg_mc, &x[i]);
+                if (quarter != 0) {
+#pragma unroll
+                    for (int c4 = 0; c4 < 8; ++c4)
+                        xs[((quarter - 1) * 8 + c4) * 32 + lane] =
+                            make_float4(x[4 * c4], x[4 * c4 + 1], x[4 * c4 + 2], x[4 * c4 + 3]);
+                }
+                named_bar_sync(2 + wg, 128);                 // weights of columns 32..127 are in shared memory
+                if (quarter == 0) {
+#pragma unroll
+                    for (int k = 0; k < 24; ++k) {
+                        const float4 v4 = xs[k * 32 + lane];
+                        x[32 + 4 * k] = v4.x;
+                        x[32 + 4 * k + 1] = v4.y;
+                        x[32 + 4 * k + 2] = v4.z;
+                        x[32 + 4 * k + 3] = v4.w;
+                    }
+                    RowSum4 rs_lo, rs_hi;
+                    rs_lo.reset();
+                    rs_hi.reset();
+                    uint32_t pk[64];
+#pragma unroll
+                    for (int i = 0; i < 64; i += 8) softmax_sum_pack8(&x[i], rs_lo, &pk[i >> 1]);
+                    tmem_st32(tp, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+#pragma unroll
+                    for (int i = 0; i < 64; i += 8) softmax_sum_pack8(&x[64 + i], rs_hi, &pk[32 + (i >> 1)]);
+                    tmem_st32(tp + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+                    const float alpha = softmax_alpha(m_old, m_new, c);
+                    if (it > 0 && !chunk_start) {
+                        wait_tile_done(it - 1);
+                        l_old_lo = st_l[lane];
+                        l_old_hi = st_l[128 + lane];
+                    }
+                    m_own = m_new;
+                    l_own_lo = __fmaf_rn(l_old_lo, alpha, rs_lo.total());
+                    l_own_hi = __fmaf_rn(l_old_hi, alpha, rs_hi.total());
+                    st_l[lane] = l_own_lo;
+                    st_l[128 + lane] = l_own_hi;
+                    if (fold_now) {
+                        wait_pv(it - 1);
+                        write_partial_ml(chunk_of(it - 1), m_prev, l_prev_lo, l_prev_hi);
+                        write_partial_o(chunk_of(it - 1), 0, D);
+                    } else if (!chunk_start && !__all_sync(0xffffffffu, alpha == 1.0f)) {
+                        wait_pv(it - 1);
+                        const uint32_t to = tlane + col_o_of(it);
+#pragma unroll
+                        for (int cc = 0; cc < D / 32; ++cc) {
+                            uint32_t v[32];
+                            tmem_ld32(to + 32 * cc, v);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
+                            tmem_st32(to + 32 * cc, v);
+                        }
+                    }
+                    tmem_wait_st();
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_pfull + 8 * wg);
+            }
+            // ---- the last chunk's partial: state by warp 0 of the warpgroup that owned the last
+            // tile, accumulator columns half by each warpgroup's warp 0
+            if (wg == (last & 1)) {
+                wait_pv(last);
+                if (quarter == 0) write_partial_ml(chunk_of(last), m_own, l_own_lo, l_own_hi);
+                tc_fence_before();
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            tc_fence_after();
+            if (quarter == 0) write_partial_o(chunk_of(last), DH * wg, DH);
+        } else if (pair) {
             // ---- paired mode: this warpgroup keeps the rows of one query tile (wg 0: tile B = T0,
             // wg 1: tile A = T1) through all of that tile's KV tiles; nothing is handed over.
             const int Tq = wg ? T1 : T0;
@@ -604,7 +800,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 // state handed over by the thread that processed tile it-1
                 float m_old = -CUDART_INF_F, l_old_lo = 0.0f, l_old_hi = 0.0f;
                 float m_prev = 0.0f, l_prev_lo = 0.0f, l_prev_hi = 0.0f;   // finished chunk, if any
-                const bool fold_now = (MODE != MODE_DECODE) && chunk_start && it > 0;
+                const bool fold_now = chunk_start && it > 0;     // a finished chunk precedes this tile
                 if (it > 0) {
                     mbar_wait(bar_m, (it - 1) & 1, abort_word, p.dev_status);
                     if (fold_now) {
@@ -646,7 +842,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 st_l[128 + r] = l_own_hi;
                 if (fold_now) {
                     wait_pv(it - 1);
-                    fold_chunk(chunk_of(it - 1), m_prev, l_prev_lo, l_prev_hi, true);
+                    if (MODE == MODE_DECODE) {
+                        write_partial_ml(chunk_of(it - 1), m_prev, l_prev_lo, l_prev_hi);
+                        write_partial_o(chunk_of(it - 1), 0, D);
+                    } else {
+                        fold_chunk(chunk_of(it - 1), m_prev, l_prev_lo, l_prev_hi, true);
+                    }
                 } else if (!chunk_start && !__all_sync(0xffffffffu, alpha == 1.0f)) {
                     // rescale the chunk accumulator of this row
                     wait_pv(it - 1);
@@ -680,13 +881,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             wait_pv(last);
             if (active) {
                 if (MODE == MODE_DECODE) {
-                    if (r < p.G) {
-                        const long long slot =
-                            (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk;
-                        p.part_ml[4 * slot] = m_own;
-                        p.part_ml[4 * slot + 1] = l_own_lo;
-                        p.part_ml[4 * slot + 2] = l_own_hi;
-                    }
+                    write_partial_ml(chunk_of(last), m_own, l_own_lo, l_own_hi);
                 } else {
                     fold_chunk(chunk_of(last), m_own, l_own_lo, l_own_hi, true);
                     const float Ltot = finalize_l(Lg_lo, Lg_hi);
@@ -702,21 +897,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // both warpgroups write half of the output columns each
         if (active) {
             if (MODE == MODE_DECODE) {
-#pragma unroll
-                for (int cc = 0; cc < DH / 32; ++cc) {
-                    uint32_t v[32];
-                    tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, v);
-                    tmem_wait_ld();
-                    if (r < p.G) {
-                        const long long slot =
-                            (static_cast<long long>(seq) * p.Hq + head + r) * p.nchunk_max + chunk;
-                        float4* dst = reinterpret_cast<float4*>(p.part_o + slot * D + DH * wg + 32 * cc);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                                 __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-                    }
-                }
+                write_partial_o(chunk_of(last), DH * wg, DH);
             } else {
                 const float inv = st_m[r];
                 const int e_row0 = meta[0], e_lo = meta[1], e_hi = meta[2];

@@ -123,20 +123,27 @@ __device__ __forceinline__ void add_rn_x2(float& a0, float& a1, float b0, float 
         : "f"(b0), "f"(b1));
 }
 // Weights and half-row sum of 8 consecutive columns (chains 0,0,1,1,2,2,3,3): every chain still
-// receives its columns in ascending order, two chains per packed add.
-__device__ __forceinline__ void softmax_p8(const uint32_t* s8, float c, float neg_mc, RowSum4& rs, uint32_t* pk4) {
-    float x[8];
+// receives its columns in ascending order, two chains per packed add.  The two steps are also
+// available separately: decode computes the weights of a row on four warps and sums on one.
+__device__ __forceinline__ void softmax_x8(const uint32_t* s8, float c, float neg_mc, float* x) {
 #pragma unroll
     for (int i = 0; i < 8; i += 2)
         fma_rn_x2(x[i], x[i + 1], __uint_as_float(s8[i]), __uint_as_float(s8[i + 1]), c, neg_mc);
 #pragma unroll
     for (int i = 0; i < 8; ++i) x[i] = ex2_ftz(x[i]);
+}
+__device__ __forceinline__ void softmax_sum_pack8(const float* x, RowSum4& rs, uint32_t* pk4) {
     add_rn_x2(rs.a[0], rs.a[1], x[0], x[2]);
     add_rn_x2(rs.a[2], rs.a[3], x[4], x[6]);
     add_rn_x2(rs.a[0], rs.a[1], x[1], x[3]);
     add_rn_x2(rs.a[2], rs.a[3], x[5], x[7]);
 #pragma unroll
     for (int i = 0; i < 4; ++i) pk4[i] = pack_bf16x2(x[2 * i], x[2 * i + 1]);
+}
+__device__ __forceinline__ void softmax_p8(const uint32_t* s8, float c, float neg_mc, RowSum4& rs, uint32_t* pk4) {
+    float x[8];
+    softmax_x8(s8, c, neg_mc, x);
+    softmax_sum_pack8(x, rs, pk4);
 }
 
 // exponent argument of one score: s * c - mc, one fused multiply-add.

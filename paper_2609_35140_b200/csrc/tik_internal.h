@@ -36,6 +36,7 @@ struct AttnParams {
     float* part_o;               // decode: [B][Hq][nchunk_max][d]
     float* part_ml;              // decode: [B][Hq][nchunk_max][4] = m, l_lo, l_hi, unused
     int nchunk_max;
+    int cpc;                     // decode: consecutive chunks streamed by one CTA
     int* dev_status;
     int lookahead;               // train / prefill: block distance of the query-tile L2 prefetch
 };
@@ -44,6 +45,16 @@ struct AttnParams {
 cudaError_t launch_attn(int d, int mode, dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                         const CUtensorMap& tmV, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_combine(int d, const AttnParams& p, int B, cudaStream_t stream);
+
+// Decode: how many consecutive chunks one CTA streams.  A CTA's set-up and drain cost about a
+// third of one chunk's streaming time, so several chunks per CTA pay as long as the grid still
+// covers every SM several times over.  Chunk partials do not depend on this choice.
+inline int decode_chunks_per_cta(long long B, int Hkv, int nchunk, int sm_count) {
+    const long long want = 4ll * (sm_count > 0 ? sm_count : 148);
+    for (int c = 4; c > 1; --c)
+        if (c <= nchunk && B * Hkv * ((nchunk + c - 1) / c) >= want) return c;
+    return 1;
+}
 cudaError_t launch_kv_write(const void* k_new, const void* v_new, const int32_t* cu_new,
                             const int32_t* ctx_lens, void* k_cache, void* v_cache,
                             const int32_t* block_table, int max_blocks, int S, int64_t total_new,

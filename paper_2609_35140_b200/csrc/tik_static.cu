@@ -138,6 +138,7 @@ extern "C" tik_status tik_attn_decode_static(const void* q, void* o, float* lse,
     // The library's own flag word keeps the last call's flags; a stale "wait expired" would
     // make every later kernel bail out, so it is cleared (stream-ordered) before each use.
     if (!dev_flags) e = cudaMemsetAsync(s->flags, 0, sizeof(int), st);
+    p.cpc = 1;
     if (e == cudaSuccess) e = launch_attn(d, 2, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st);
     if (e == cudaSuccess) e = launch_combine(d, p, B, st);
     return e == cudaSuccess ? TIK_OK : TIK_ERR_CUDA;
