@@ -35,6 +35,7 @@ WORKLOADS = {
     "d64_page32": lambda: synth.custom_workload([33, 250], [95, 140], 6, 3, 64, 32),
     "d128_page16_g1": lambda: synth.custom_workload([70], [186], 2, 2, 128, 16),
     "d128_page128_g16": lambda: synth.custom_workload([128, 5], [130, 250], 16, 1, 128, 128),
+    "d64_page64_g32": lambda: synth.custom_workload([40, 130], [100, 30], 32, 1, 64, 64),
 }
 
 

@@ -230,3 +230,31 @@ def test_bad_block_table_entry_is_flagged_not_fatal(tik, case):
     assert tik.device_status() & tik.DEV_BAD_BLOCK
     assert torch.equal(bits(o[0]), bits(o_train[rows[0]]))            # the other slot is unaffected
     assert bool(torch.isfinite(o.float()).all())
+
+
+def test_decode_with_several_chunks_per_cta(tik):
+    """A large decode batch lets one CTA stream up to four consecutive 2048-key chunks; a small
+    one gets a CTA per chunk.  The chunk partials, and so every output bit, must not depend on it."""
+    rng = np.random.default_rng(77)
+    lens = [int(x) for x in rng.integers(2100, 6200, 150)]
+    lens[0], lens[1], lens[2] = 8192, 2048, 2049          # exactly four chunks, one chunk, one chunk + one key
+    w = synth.custom_workload([1] * len(lens), [L - 1 for L in lens], 4, 4, 64, 64, index=33)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    o_train = tik.tik_attn_train_fwd(q, k, v, cu, max(w.seq_lens), w.softmax_scale)
+    layout = synth.make_paged_layout(w)
+    kc, vc, bt = _full_cache(tik, w, k, v, cu, layout)
+    seqs = list(range(w.S))
+    for frac in (1.0, 0.55):
+        pos = [max(1, int(L * frac)) - 1 for L in lens]
+        rows, o = _decode_rows(tik, w, q, kc, vc, bt, seqs, pos)
+        assert count_diff(o, o_train[rows]) == 0, frac
+        # the same rows decoded three at a time (one CTA per chunk)
+        for s0 in (0, 60):
+            sub = seqs[s0:s0 + 3]
+            rows3, o3 = _decode_rows(tik, w, q, kc, vc, bt, sub, [pos[s] for s in sub])
+            assert count_diff(o3, o_train[rows3]) == 0
+    ref = oracle.attn_rows(q[rows[:4], 1].float().cpu().numpy(),
+                           np.concatenate([k[int(cu[s]):int(cu[s + 1]), 1].float().cpu().numpy() for s in range(4)]),
+                           np.concatenate([v[int(cu[s]):int(cu[s + 1]), 1].float().cpu().numpy() for s in range(4)]),
+                           [int(cu[s]) for s in range(4)], [p + 1 for p in pos[:4]], w.softmax_scale)[0]
+    assert np.abs(o[:4, 1].float().cpu().numpy() - ref).max() <= ATTN_TOL
