@@ -156,3 +156,31 @@ def log_softmax_row(hidden_row, W, inv_temperature: float = 1.0, f32: bool = Fal
         ctypes.c_double(inv_temperature), _p(out))
     assert rc == 0
     return out
+
+
+def norm_rope(x, w, eps: float, cos_sin, pos, f32: bool = False):
+    """x [T,H,d], w [d] or None, cos_sin [max_pos,d] (cos | sin), pos [T] -> RMSNorm then NeoX RoPE, [T,H,d]."""
+    x, cos_sin, pos = _f32(x), _f32(cos_sin), _i64(pos)
+    T, H, d = x.shape
+    assert d % 2 == 0 and cos_sin.shape[1] == d and pos.shape == (T,)
+    wp = None
+    if w is not None:
+        w = _f32(w)
+        assert w.shape == (d,)
+        wp = _p(w)
+    dt, sfx = _real(f32)
+    out = np.empty((T, H, d), dtype=dt)
+    rc = getattr(lib(), "oracle_norm_rope" + sfx)(
+        _p(x), wp, ctypes.c_double(eps), _p(cos_sin), ctypes.c_int64(cos_sin.shape[0]), _p(pos),
+        ctypes.c_int64(T), ctypes.c_int(H), ctypes.c_int(d), _p(out))
+    assert rc == 0, "position outside the cos/sin table"
+    return out
+
+
+def paged_scatter(rows, pos, block_table_row, page_size: int, cache):
+    """Indexed KV-cache write as its plain definition: token i of one sequence, at position pos[i],
+    goes to cache[block_table_row[pos[i] // page_size], :, pos[i] % page_size, :].  rows [n,Hkv,d];
+    cache [num_pages,Hkv,page_size,d] is modified in place and returned."""
+    for i, p in enumerate(pos):
+        cache[int(block_table_row[int(p) // page_size]), :, int(p) % page_size, :] = rows[i]
+    return cache

@@ -1,4 +1,5 @@
-/* CPU oracle for causal grouped-query attention and token log-probability.
+/* CPU oracle for causal grouped-query attention, token log-probability and the pre-attention
+ * step (RMSNorm -> NeoX RoPE; the indexed cache write is a numpy index copy in __init__.py).
  *
  * TEST INFRASTRUCTURE ONLY.  Only the tests, the smoke check and the
  * benchmark's CPU-baseline leg may load this library.  It shares no code,
@@ -15,7 +16,11 @@
  * value; causality; GQA equals MHA with repeated KV; key-shift invariance;
  * brute-force loops on tiny inputs; library attention / log_softmax on a
  * textbook case; zero weights give -ln V; one-hot logits in closed form;
- * paged storage equals packed storage.
+ * paged storage equals packed storage.  Pre-attention step (tests/test_oracle_prep.py): RoPE as
+ * numpy's complex product on the pairs (i, i + d/2); position 0 is the identity; norms kept and
+ * scores a function of relative position; RMSNorm against closed forms and torch's rms_norm in
+ * fp64; norm before rotation; the cos/sin table against hand values and the angle-addition
+ * identity; the cache write against its index definition.
  */
 #include <math.h>
 #include <stdint.h>

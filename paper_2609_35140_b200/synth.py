@@ -251,6 +251,26 @@ def make_logprob_inputs(w: Workload, device="cpu", T: Optional[int] = None, seed
     return hidden, W, target.to(torch.int32)
 
 
+def make_rope_table(max_pos: int, d: int, base: float = 1.0e6, device="cpu") -> torch.Tensor:
+    """The cos/sin table the pre-attention step takes as an input: fp32 [max_pos, d], row p =
+    cos(p * theta_i) for i < d/2, then sin(p * theta_i), with theta_i = base^(-2i/d) (angles in fp64,
+    rounded once).  base 1e6 is the Qwen2.5 / Qwen3 setting."""
+    i = torch.arange(d // 2, dtype=torch.float64)
+    theta = torch.pow(torch.tensor(float(base), dtype=torch.float64), -2.0 * i / d)
+    ang = torch.arange(max_pos, dtype=torch.float64)[:, None] * theta[None, :]
+    return torch.cat([torch.cos(ang), torch.sin(ang)], dim=1).to(torch.float32).to(device)
+
+
+def make_norm_weights(w: Workload, device="cpu", seed_offset: int = 0):
+    """Per-head RMSNorm weights for Q and K, bf16 [d] each, around one (trained norm weights
+    stay close to their initial value of one)."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(w.seed + 7919 + seed_offset)
+    wq = (1.0 + 0.2 * torch.randn(w.d, generator=gen)).to(torch.bfloat16).to(device)
+    wk = (1.0 + 0.2 * torch.randn(w.d, generator=gen)).to(torch.bfloat16).to(device)
+    return wq, wk
+
+
 def sample_rows(w: Workload, n_random: int, seed_offset: int = 1) -> List[Tuple[int, int, int]]:
     """(sequence, query head, position) rows worth checking one by one: every
     sequence's first and last row, rows around the 128-key tile, page and
