@@ -47,6 +47,7 @@ typedef int tik_status;
 #define TIK_DEV_BAD_BLOCK 1        /* block-table entry outside [0,num_pages): page read as zeros */
 #define TIK_DEV_BAD_TARGET 2       /* target id outside [0,V): logprob = NaN */
 #define TIK_DEV_WAIT_EXPIRED 4     /* an in-kernel bounded wait ran out (outputs invalid) */
+#define TIK_DEV_BAD_POSITION 8     /* token position outside the cos/sin table: token left untouched */
 
 #define TIK_OP_ATTN_TRAIN_FWD 0
 #define TIK_OP_ATTN_PREFILL 1
@@ -96,6 +97,38 @@ tik_status tik_kv_cache_write(tik_ctx* ctx, const void* k_new, const void* v_new
                               void* k_cache, void* v_cache, const int32_t* block_table,
                               int max_blocks, int S, int64_t total_new, int Hkv, int d,
                               int page_size, int num_pages, void* stream);
+
+/* Pre-attention step in one pass: per-head RMSNorm of Q and K, NeoX rotary embedding of Q and K,
+ * indexed write of K and V into the paged cache.  The paper's operator table (Sec. 6, operator
+ * correctness) lists Q RMSNorm, K RMSNorm, NeoX RoPE (Q, K) and the indexed KV-cache write as
+ * unified operators verified bitwise between full-sequence and token-wise use; it gives no
+ * formulas, so the textbook definitions apply, and the fusion and the order norm -> rotation ->
+ * write (the Qwen3 layer order) are this library's choice.  Per (token, head) vector x of length d:
+ *   y_i = x_i * rsqrt(mean_j x_j^2 + eps) * w_i                     (skipped when the weight is NULL)
+ *   z_i = y_i cos_i - y_{i+d/2} sin_i,  z_{i+d/2} = y_{i+d/2} cos_i + y_i sin_i   for i < d/2
+ * with (cos_i, sin_i) = cos_sin[pos][i], cos_sin[pos][d/2 + i]: a caller-built fp32 table
+ * [max_pos][d] of cos(p theta_i) | sin(p theta_i) (device memory).  Arithmetic is fp32 with one
+ * rounding to bf16 at the end; a vector's result depends on that vector, the weight, eps and its
+ * table row only, never on the other tokens of the call.
+ *   q [total_new][Hq][d], k [total_new][Hkv][d]: bf16, device, overwritten in place
+ *   v [total_new][Hkv][d]: read only; may be NULL when there is no cache
+ *   q_weight, k_weight: bf16 [d], device, each may be NULL
+ *   token i of sequence s (rows cu_seqlens_new[s]..) has position ctx_lens[s] - n_s + i, where
+ *   ctx_lens[s] is the context length AFTER this step; ctx_lens == NULL means positions start at 0
+ *   (whole sequences, the policy-update forward)
+ *   k_cache, v_cache [num_pages][Hkv][page_size][d]: both NULL = no cache write (then block_table
+ *   is ignored); otherwise rotated K and V go to page block_table[s][pos / page_size], row
+ *   pos % page_size, exactly the bf16 values written back to k / read from v
+ * Device flags: TIK_DEV_BAD_POSITION (position outside [0, max_pos): the token's q, k and cache
+ * rows are left untouched), TIK_DEV_BAD_BLOCK (bad table entry: q and k are still transformed, the
+ * cache is not written).  Needs no workspace; launches one kernel on `stream`. */
+tik_status tik_qk_norm_rope_kv_write(tik_ctx* ctx, void* q, void* k, const void* v,
+                                     const void* q_weight, const void* k_weight, float eps,
+                                     const float* cos_sin, int max_pos,
+                                     const int32_t* cu_seqlens_new, const int32_t* ctx_lens,
+                                     void* k_cache, void* v_cache, const int32_t* block_table,
+                                     int max_blocks, int S, int64_t total_new, int Hq, int Hkv,
+                                     int d, int page_size, int num_pages, void* stream);
 
 /* Rollout prefill attention (paper Sec. 4.1: the full-sequence entry point applied to a
  * prompt) against the paged cache, which must already hold the keys/values of positions

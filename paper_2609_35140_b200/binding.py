@@ -17,7 +17,7 @@ from . import build as _build
 
 OK = 0
 OP_ATTN_TRAIN_FWD, OP_ATTN_PREFILL, OP_ATTN_DECODE, OP_TOKEN_LOGPROB = 0, 1, 2, 3
-DEV_BAD_BLOCK, DEV_BAD_TARGET, DEV_WAIT_EXPIRED = 1, 2, 4
+DEV_BAD_BLOCK, DEV_BAD_TARGET, DEV_WAIT_EXPIRED, DEV_BAD_POSITION = 1, 2, 4, 8
 
 _lib = None
 _ctx = {}
@@ -57,12 +57,15 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
                                      i32, i32, i32, f32, vp]
     lib.tik_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32,
                                     f32, vp, sz, vp]
+    lib.tik_qk_norm_rope_kv_write.argtypes = [vp, vp, vp, vp, vp, vp, f32, vp, i32, vp, vp, vp, vp, vp, i32, i32,
+                                              i64, i32, i32, i32, i32, i32, vp]
     lib.tik_token_logprob.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, f32, vp, sz, vp]
     lib.tik_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
                                            i32, f32, vp, vp]
     lib.tik_attn_decode_static.restype = i32
     for name in ("tik_create", "tik_destroy", "tik_device_status", "tik_attn_train_fwd",
-                 "tik_kv_cache_write", "tik_attn_prefill", "tik_attn_decode", "tik_token_logprob"):
+                 "tik_kv_cache_write", "tik_attn_prefill", "tik_attn_decode", "tik_token_logprob",
+                 "tik_qk_norm_rope_kv_write"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -147,6 +150,25 @@ def tik_kv_cache_write(k_new, v_new, cu_seqlens_new, ctx_lens, k_cache, v_cache,
                                    _ptr(k_cache, bf), _ptr(v_cache, bf),
                                    _ptr(block_table, torch.int32), block_table.shape[1],
                                    ctx_lens.numel(), k_new.shape[0], Hkv, d, page, num_pages, _stream())
+    _check(rc, ctx)
+
+
+def tik_qk_norm_rope_kv_write(q, k, v, q_weight, k_weight, eps: float, cos_sin, cu_seqlens_new,
+                              ctx_lens=None, k_cache=None, v_cache=None, block_table=None):
+    """Per-head RMSNorm (weights may be None) and NeoX RoPE of q [n,Hq,d] and k [n,Hkv,d] in place;
+    with caches, rotated K and V also go to the pages.  cos_sin fp32 [max_pos,d]."""
+    ctx = context()
+    bf = torch.bfloat16
+    n, Hq, d = q.shape
+    Hkv = k.shape[1]
+    page = k_cache.shape[2] if k_cache is not None else 0
+    num_pages = k_cache.shape[0] if k_cache is not None else 0
+    rc = load().tik_qk_norm_rope_kv_write(
+        ctx, _ptr(q, bf), _ptr(k, bf), _ptr(v, bf), _ptr(q_weight, bf), _ptr(k_weight, bf), float(eps),
+        _ptr(cos_sin, torch.float32), cos_sin.shape[0], _ptr(cu_seqlens_new, torch.int32),
+        _ptr(ctx_lens, torch.int32), _ptr(k_cache, bf), _ptr(v_cache, bf), _ptr(block_table, torch.int32),
+        block_table.shape[1] if block_table is not None else 0, cu_seqlens_new.numel() - 1, n, Hq, Hkv, d,
+        page, num_pages, _stream())
     _check(rc, ctx)
 
 

@@ -335,6 +335,53 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_decode");
 }
 
+tik_status tik_qk_norm_rope_kv_write(tik_ctx* ctx, void* q, void* k, const void* v, const void* q_weight,
+                                     const void* k_weight, float eps, const float* cos_sin, int max_pos,
+                                     const int32_t* cu_seqlens_new, const int32_t* ctx_lens, void* k_cache,
+                                     void* v_cache, const int32_t* block_table, int max_blocks, int S,
+                                     int64_t total_new, int Hq, int Hkv, int d, int page_size, int num_pages,
+                                     void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (S < 0 || total_new < 0 || max_pos < 0 || max_blocks < 0 || num_pages < 0)
+        return fail(ctx, TIK_ERR_INVALID_ARG, "negative size");
+    if (Hq <= 0 || Hkv <= 0) return fail(ctx, TIK_ERR_INVALID_ARG, "Hq and Hkv must be positive");
+    if (!(eps >= 0.0f) || !std::isfinite(eps)) return fail(ctx, TIK_ERR_INVALID_ARG, "eps must be finite and >= 0");
+    if (d != 64 && d != 128) return fail(ctx, TIK_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    const bool cache = k_cache != nullptr || v_cache != nullptr;
+    if (cache && !page_ok(page_size)) return fail(ctx, TIK_ERR_UNSUPPORTED, "page_size must be 16, 32, 64 or 128");
+    if (S == 0 || total_new == 0) return TIK_OK;
+    if (!q || !k || !cos_sin || !cu_seqlens_new || max_pos == 0) return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (cache && (!k_cache || !v_cache || !v || !block_table || num_pages == 0))
+        return fail(ctx, TIK_ERR_INVALID_ARG, "cache write needs k_cache, v_cache, v and block_table");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache) ||
+        !aligned16(q_weight) || !aligned16(k_weight) || !aligned16(cos_sin))
+        return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (total_new >= (1ll << 31)) return fail(ctx, TIK_ERR_UNSUPPORTED, "total_new must be < 2^31");
+    PrepParams p{};
+    p.q = static_cast<__nv_bfloat16*>(q);
+    p.k = static_cast<__nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.q_weight = static_cast<const __nv_bfloat16*>(q_weight);
+    p.k_weight = static_cast<const __nv_bfloat16*>(k_weight);
+    p.eps = eps;
+    p.cos_sin = cos_sin;
+    p.max_pos = max_pos;
+    p.cu_new = cu_seqlens_new;
+    p.ctx_lens = ctx_lens;
+    p.k_cache = static_cast<__nv_bfloat16*>(k_cache);
+    p.v_cache = static_cast<__nv_bfloat16*>(v_cache);
+    p.block_table = block_table;
+    p.max_blocks = max_blocks;
+    p.S = S;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.page_size = page_size;
+    p.num_pages = num_pages;
+    p.dev_status = ctx->dev_status;
+    cudaError_t e = launch_prep(d, p, total_new, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_qk_norm_rope_kv_write");
+}
+
 tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_head, const int32_t* target_ids,
                              float* logprob, float* lse, int64_t T, int H, int V, float inv_temperature, void* ws,
                              size_t ws_bytes, void* stream) {

@@ -189,4 +189,33 @@ __device__ __forceinline__ float lp_lse(float M, float L) {
     return __fadd_rn(M, __fmul_rn(log2f(L), LN2_F));
 }
 
+// ---- pre-attention step: per-head RMSNorm and NeoX rotation of one (token, head) vector ------
+// One warp holds the vector: lane l has EP elements of the first half and their partners i + d/2
+// (d = 128: elements 2l, 2l+1; d = 64: element l).  Sum of squares: per lane a fused chain in the
+// order lo[0], lo[1], hi[0], hi[1], then a butterfly over lane distances 16, 8, 4, 2, 1 (both
+// partners of an exchange add the same two numbers, so every lane ends with the same total).
+template <int EP>
+__device__ __forceinline__ float prep_sum_squares(const float* lo, const float* hi) {
+    float part = __fmul_rn(lo[0], lo[0]);
+#pragma unroll
+    for (int e = 1; e < EP; ++e) part = __fmaf_rn(lo[e], lo[e], part);
+#pragma unroll
+    for (int e = 0; e < EP; ++e) part = __fmaf_rn(hi[e], hi[e], part);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) part = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, off));
+    return part;
+}
+// 1 / sqrt(ss / d + eps), correctly rounded reciprocal square root of one fused multiply-add
+__device__ __forceinline__ float prep_inv_rms(float ss, float inv_d, float eps) {
+    return __frsqrt_rn(__fmaf_rn(ss, inv_d, eps));
+}
+__device__ __forceinline__ float prep_norm(float x, float inv, float w) { return __fmul_rn(__fmul_rn(x, inv), w); }
+// (lo, hi) <- (lo cos - hi sin, hi cos + lo sin): four products and two sums, none fused
+__device__ __forceinline__ void prep_rotate(float& lo, float& hi, float cs, float sn) {
+    const float a = __fsub_rn(__fmul_rn(lo, cs), __fmul_rn(hi, sn));
+    const float b = __fadd_rn(__fmul_rn(hi, cs), __fmul_rn(lo, sn));
+    lo = a;
+    hi = b;
+}
+
 }  // namespace tik

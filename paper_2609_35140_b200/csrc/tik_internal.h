@@ -1,5 +1,6 @@
 // Host-side declarations shared by the translation units of libtik (not part of the ABI).
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -45,6 +46,25 @@ struct AttnParams {
 cudaError_t launch_attn(int d, int mode, dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                         const CUtensorMap& tmV, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_combine(int d, const AttnParams& p, int B, cudaStream_t stream);
+
+struct PrepParams {
+    __nv_bfloat16* q;            // [total_new][Hq][d], in place
+    __nv_bfloat16* k;            // [total_new][Hkv][d], in place
+    const __nv_bfloat16* v;      // [total_new][Hkv][d] or null
+    const __nv_bfloat16* q_weight;   // [d] or null (no Q norm)
+    const __nv_bfloat16* k_weight;   // [d] or null (no K norm)
+    float eps;
+    const float* cos_sin;        // [max_pos][d]: cos | sin
+    int max_pos;
+    const int32_t* cu_new;       // [S+1]
+    const int32_t* ctx_lens;     // [S] context after the write, or null (positions start at 0)
+    __nv_bfloat16* k_cache;      // [num_pages][Hkv][page_size][d] or null (no cache write)
+    __nv_bfloat16* v_cache;
+    const int32_t* block_table;
+    int max_blocks, S, Hq, Hkv, page_size, num_pages;
+    int* dev_status;
+};
+cudaError_t launch_prep(int d, const PrepParams& p, int64_t total_new, cudaStream_t stream);
 
 // Decode: how many consecutive chunks one CTA streams.  A CTA's set-up and drain cost about a
 // third of one chunk's streaming time, so several chunks per CTA pay as long as the grid still

@@ -14,6 +14,7 @@ constexpr unsigned long long TIK_WAIT_LIMIT_NS = 2000000000ull;  // 2 s per wait
 constexpr int TIK_DEV_BAD_BLOCK = 1;      // block-table entry outside [0, num_pages)
 constexpr int TIK_DEV_BAD_TARGET = 2;     // target id outside [0, V)
 constexpr int TIK_DEV_WAIT_EXPIRED = 4;   // a bounded wait ran out
+constexpr int TIK_DEV_BAD_POSITION = 8;   // token position outside the cos/sin table
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
