@@ -377,6 +377,7 @@ tik_status tik_qk_norm_rope_kv_write(tik_ctx* ctx, void* q, void* k, const void*
     p.Hkv = Hkv;
     p.page_size = page_size;
     p.num_pages = num_pages;
+    p.total_new = total_new;
     p.dev_status = ctx->dev_status;
     cudaError_t e = launch_prep(d, p, total_new, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_qk_norm_rope_kv_write");

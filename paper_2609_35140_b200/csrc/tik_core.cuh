@@ -190,10 +190,10 @@ __device__ __forceinline__ float lp_lse(float M, float L) {
 }
 
 // ---- pre-attention step: per-head RMSNorm and NeoX rotation of one (token, head) vector ------
-// One warp holds the vector: lane l has EP elements of the first half and their partners i + d/2
-// (d = 128: elements 2l, 2l+1; d = 64: element l).  Sum of squares: per lane a fused chain in the
-// order lo[0], lo[1], hi[0], hi[1], then a butterfly over lane distances 16, 8, 4, 2, 1 (both
-// partners of an exchange add the same two numbers, so every lane ends with the same total).
+// Sixteen lanes hold the vector: lane l has EP = d/32 consecutive elements of the first half and
+// their partners i + d/2.  Sum of squares: per lane a fused chain over lo[0..EP), then hi[0..EP),
+// then a butterfly over lane distances 8, 4, 2, 1 (both partners of an exchange add the same two
+// numbers, so all sixteen lanes end with the same total).
 template <int EP>
 __device__ __forceinline__ float prep_sum_squares(const float* lo, const float* hi) {
     float part = __fmul_rn(lo[0], lo[0]);
@@ -202,7 +202,7 @@ __device__ __forceinline__ float prep_sum_squares(const float* lo, const float* 
 #pragma unroll
     for (int e = 0; e < EP; ++e) part = __fmaf_rn(hi[e], hi[e], part);
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) part = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, off));
+    for (int off = 8; off >= 1; off >>= 1) part = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, off));
     return part;
 }
 // 1 / sqrt(ss / d + eps), correctly rounded reciprocal square root of one fused multiply-add

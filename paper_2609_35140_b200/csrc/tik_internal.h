@@ -62,6 +62,7 @@ struct PrepParams {
     __nv_bfloat16* v_cache;
     const int32_t* block_table;
     int max_blocks, S, Hq, Hkv, page_size, num_pages;
+    long long total_new;
     int* dev_status;
 };
 cudaError_t launch_prep(int d, const PrepParams& p, int64_t total_new, cudaStream_t stream);
