@@ -37,7 +37,7 @@ METRIC = "summed_attention_ms"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch of the dominant kernel from one ncu capture (profiles/), keyed by
 # workload index; None until captured.
-NCU_TRAFFIC_BYTES = {1: 2902704600}     # logprob_kernel on workload 1: 2.872 GB read + 30.4 MB written
+NCU_TRAFFIC_BYTES = {1: 2905034344}     # logprob_kernel on workload 1: 2.872 GB read + 30.4 MB written
 
 
 def load_peaks():

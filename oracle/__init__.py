@@ -184,3 +184,44 @@ def paged_scatter(rows, pos, block_table_row, page_size: int, cache):
     for i, p in enumerate(pos):
         cache[int(block_table_row[int(p) // page_size]), :, int(p) % page_size, :] = rows[i]
     return cache
+
+
+def rmsnorm(x, w, eps: float, residual=None, f32: bool = False):
+    """x [T,H], w [H] -> y [T,H].  With residual [T,H]: s = bf16(x + residual) is normalised and
+    also returned: (y, s)."""
+    x, w = _f32(x), _f32(w)
+    T, H = x.shape
+    assert w.shape == (H,)
+    res = None if residual is None else _f32(residual)
+    dt, sfx = _real(f32)
+    y = np.empty((T, H), dtype=dt)
+    s = np.empty((T, H), dtype=np.float32) if res is not None else None
+    rc = getattr(lib(), "oracle_rmsnorm" + sfx)(_p(x), _p(res), _p(w), ctypes.c_double(eps), ctypes.c_int64(T),
+                                               ctypes.c_int(H), _p(y), _p(s))
+    assert rc == 0
+    return y if res is None else (y, s)
+
+
+def swiglu(gate_up, f32: bool = False):
+    """gate_up [T,2I] (gate | up) -> silu(gate) * up, [T,I]."""
+    gu = _f32(gate_up)
+    T, I2 = gu.shape
+    assert I2 % 2 == 0
+    dt, sfx = _real(f32)
+    out = np.empty((T, I2 // 2), dtype=dt)
+    rc = getattr(lib(), "oracle_swiglu" + sfx)(_p(gu), ctypes.c_int64(T), ctypes.c_int(I2 // 2), _p(out))
+    assert rc == 0
+    return out
+
+
+def linear(x, W, f32: bool = False):
+    """x [T,K], W [N,K] -> x @ W.T, [T,N]."""
+    x, W = _f32(x), _f32(W)
+    T, K = x.shape
+    N = W.shape[0]
+    assert W.shape[1] == K
+    dt, sfx = _real(f32)
+    y = np.empty((T, N), dtype=dt)
+    rc = getattr(lib(), "oracle_linear" + sfx)(_p(x), _p(W), ctypes.c_int64(T), ctypes.c_int(K), ctypes.c_int(N), _p(y))
+    assert rc == 0
+    return y
