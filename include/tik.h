@@ -166,6 +166,31 @@ tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_he
                              int H, int V, float inv_temperature, void* ws, size_t ws_bytes,
                              void* stream);
 
+/* Hidden RMSNorm, optionally fused with the residual add (the paper's operator table, Sec. 6:
+ * "Hidden RMSNorm", "Fused residual + RMSNorm"; no formulas are given, the textbook ones apply).
+ *   residual == NULL:  y[t] = x[t] * rsqrt(mean_j x[t][j]^2 + eps) * weight
+ *   residual != NULL:  s = bf16(x + residual) (fp32 sum rounded to bf16) is stored back to
+ *                      residual and normalised: y[t] = s * rsqrt(mean s^2 + eps) * weight,
+ *                      exactly what a bf16 add followed by the plain form gives.
+ * x, residual, y: bf16 [T][H], device; weight bf16 [H]; y may alias x.  fp32 arithmetic, one
+ * rounding of y.  A row's result depends on that row only (fixed reduction shape), not on T.
+ * H must be a multiple of 8 and <= 8192. */
+tik_status tik_rmsnorm(tik_ctx* ctx, const void* x, void* residual, const void* weight, void* y,
+                       float eps, int64_t T, int H, void* stream);
+
+/* SwiGLU on a fused gate/up projection (operator table: "Standalone SwiGLU"): row t of gate_up
+ * [T][2I] holds gate (first I columns) then up (last I); out[t][i] = silu(gate) * up with
+ * silu(g) = g / (1 + exp(-g)); bf16 in and out, fp32 arithmetic.  I must be a multiple of 8. */
+tik_status tik_swiglu(tik_ctx* ctx, const void* gate_up, void* out, int64_t T, int I, void* stream);
+
+/* Dense linear layer without bias (operator table: "Generic dense FFN"): y = x W^T with
+ * x bf16 [T][K], weight bf16 [N][K] (the nn.Linear layout), y bf16 [T][N]; fp32 accumulation over
+ * K in one fixed ascending order, one rounding to bf16.  Row t of y depends on row t of x and on
+ * weight only, so it has the same bits at T = 1 and inside any batch.  K must be a multiple of
+ * 64, N a multiple of 8.  No workspace. */
+tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, int64_t T, int K,
+                      int N, void* stream);
+
 /* Decode attention without any allocation (the paper has no counterpart; this variant
  * exists for deployments of this library).  Same arguments, kernels and output bits as
  * tik_attn_decode, but it takes no tik_ctx and no workspace: the split-KV scratch is a

@@ -59,13 +59,16 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
                                     f32, vp, sz, vp]
     lib.tik_qk_norm_rope_kv_write.argtypes = [vp, vp, vp, vp, vp, vp, f32, vp, i32, vp, vp, vp, vp, vp, i32, i32,
                                               i64, i32, i32, i32, i32, i32, vp]
+    lib.tik_rmsnorm.argtypes = [vp, vp, vp, vp, vp, f32, i64, i32, vp]
+    lib.tik_swiglu.argtypes = [vp, vp, vp, i64, i32, vp]
+    lib.tik_linear.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp]
     lib.tik_token_logprob.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, f32, vp, sz, vp]
     lib.tik_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
                                            i32, f32, vp, vp]
     lib.tik_attn_decode_static.restype = i32
     for name in ("tik_create", "tik_destroy", "tik_device_status", "tik_attn_train_fwd",
                  "tik_kv_cache_write", "tik_attn_prefill", "tik_attn_decode", "tik_token_logprob",
-                 "tik_qk_norm_rope_kv_write"):
+                 "tik_qk_norm_rope_kv_write", "tik_rmsnorm", "tik_swiglu", "tik_linear"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -170,6 +173,45 @@ def tik_qk_norm_rope_kv_write(q, k, v, q_weight, k_weight, eps: float, cos_sin, 
         block_table.shape[1] if block_table is not None else 0, cu_seqlens_new.numel() - 1, n, Hq, Hkv, d,
         page, num_pages, _stream())
     _check(rc, ctx)
+
+
+def tik_rmsnorm(x, weight, eps: float, residual=None, y: Optional[torch.Tensor] = None):
+    """RMSNorm of x [T,H] over H; with residual [T,H], residual <- bf16(x + residual) first and that
+    sum is normalised.  Returns y [T,H]."""
+    ctx = context()
+    bf = torch.bfloat16
+    T, H = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    rc = load().tik_rmsnorm(ctx, _ptr(x, bf), _ptr(residual, bf), _ptr(weight, bf), _ptr(y, bf), float(eps),
+                            T, H, _stream())
+    _check(rc, ctx)
+    return y
+
+
+def tik_swiglu(gate_up, out: Optional[torch.Tensor] = None):
+    """gate_up [T,2I] (gate | up) -> silu(gate) * up, [T,I]."""
+    ctx = context()
+    bf = torch.bfloat16
+    T, I2 = gate_up.shape
+    if out is None:
+        out = torch.empty(T, I2 // 2, dtype=bf, device=gate_up.device)
+    rc = load().tik_swiglu(ctx, _ptr(gate_up, bf), _ptr(out, bf), T, I2 // 2, _stream())
+    _check(rc, ctx)
+    return out
+
+
+def tik_linear(x, weight, y: Optional[torch.Tensor] = None):
+    """x [T,K] @ weight[N,K]^T -> y [T,N] (bf16, fp32 accumulation)."""
+    ctx = context()
+    bf = torch.bfloat16
+    T, K = x.shape
+    N = weight.shape[0]
+    if y is None:
+        y = torch.empty(T, N, dtype=bf, device=x.device)
+    rc = load().tik_linear(ctx, _ptr(x, bf), _ptr(weight, bf), _ptr(y, bf), T, K, N, _stream())
+    _check(rc, ctx)
+    return y
 
 
 def tik_attn_prefill(q, cu_seqlens_q, ctx_lens, k_cache, v_cache, block_table, max_q_len: int,

@@ -425,4 +425,69 @@ tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_he
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_token_logprob");
 }
 
+tik_status tik_rmsnorm(tik_ctx* ctx, const void* x, void* residual, const void* weight, void* y, float eps,
+                       int64_t T, int H, void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (T < 0 || H <= 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative or zero size");
+    if (!(eps >= 0.0f) || !std::isfinite(eps)) return fail(ctx, TIK_ERR_INVALID_ARG, "eps must be finite and >= 0");
+    if (H % 8 != 0 || H > 8192) return fail(ctx, TIK_ERR_UNSUPPORTED, "H must be a multiple of 8 and <= 8192");
+    if (T == 0) return TIK_OK;
+    if (!x || !weight || !y) return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(x) || !aligned16(residual) || !aligned16(weight) || !aligned16(y))
+        return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (T >= (1ll << 31)) return fail(ctx, TIK_ERR_UNSUPPORTED, "T must be < 2^31");
+    NormParams p{};
+    p.x = static_cast<const __nv_bfloat16*>(x);
+    p.residual = static_cast<__nv_bfloat16*>(residual);
+    p.weight = static_cast<const __nv_bfloat16*>(weight);
+    p.y = static_cast<__nv_bfloat16*>(y);
+    p.eps = eps;
+    p.T = T;
+    p.H = H;
+    cudaError_t e = launch_rmsnorm(p, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_rmsnorm");
+}
+
+tik_status tik_swiglu(tik_ctx* ctx, const void* gate_up, void* out, int64_t T, int I, void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (T < 0 || I <= 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative or zero size");
+    if (I % 8 != 0) return fail(ctx, TIK_ERR_UNSUPPORTED, "I must be a multiple of 8");
+    if (T == 0) return TIK_OK;
+    if (!gate_up || !out) return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(gate_up) || !aligned16(out)) return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (T * (I / 8) >= (1ll << 39)) return fail(ctx, TIK_ERR_UNSUPPORTED, "T * I too large");
+    cudaError_t e = launch_swiglu(gate_up, out, T, I, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_swiglu");
+}
+
+tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, int64_t T, int K, int N,
+                      void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (T < 0 || K <= 0 || N <= 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative or zero size");
+    if (K % 64 != 0) return fail(ctx, TIK_ERR_UNSUPPORTED, "K must be a multiple of 64");
+    if (N % 8 != 0) return fail(ctx, TIK_ERR_UNSUPPORTED, "N must be a multiple of 8");
+    if (T == 0) return TIK_OK;
+    if (!x || !weight || !y) return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(x) || !aligned16(weight) || !aligned16(y)) return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (T >= (1ll << 31) - 128) return fail(ctx, TIK_ERR_UNSUPPORTED, "T must be < 2^31 - 128");
+    CUtensorMap tmA, tmB;
+    std::string err;
+    uint64_t ad[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(T)};
+    uint64_t bd[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(N)};
+    uint64_t st1[1] = {static_cast<uint64_t>(K) * 2};
+    uint32_t box[2] = {64, 128};
+    uint32_t boxB[2] = {64, 256};
+    if (!make_tmap_bf16(ctx, &tmA, x, 2, ad, st1, box, &err) || !make_tmap_bf16(ctx, &tmB, weight, 2, bd, st1, boxB, &err))
+        return fail(ctx, TIK_ERR_CUDA, err.c_str());
+    LinearParams p{};
+    p.y = static_cast<__nv_bfloat16*>(y);
+    p.T = T;
+    p.K = K;
+    p.N = N;
+    p.nsuper = (N + 1023) / 1024;
+    p.dev_status = ctx->dev_status;
+    cudaError_t e = launch_linear(tmA, tmB, p, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_linear");
+}
+
 }  // extern "C"

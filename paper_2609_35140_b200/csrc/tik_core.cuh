@@ -218,4 +218,27 @@ __device__ __forceinline__ void prep_rotate(float& lo, float& hi, float cs, floa
     hi = b;
 }
 
+// ---- hidden RMSNorm (optionally fused with the residual add) and SwiGLU ----------------------
+// Row of H elements on 128 threads: thread t holds the 8-element vectors t, t + 128, ... in
+// ascending order.  Residual form: s = bf16(fp32(x) + fp32(res)) is what is stored and what is
+// normalised.  Sum of squares: per thread one fused chain over its elements in that order, a
+// butterfly over lane distances 16..1, then the four warp totals as (w0 + w1) + (w2 + w3).
+__device__ __forceinline__ float hn_residual_sum(float x, float res) {
+    return __bfloat162float(__float2bfloat16_rn(__fadd_rn(x, res)));
+}
+__device__ __forceinline__ float hn_warp_total(float part) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) part = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, off));
+    return part;
+}
+__device__ __forceinline__ float hn_block_total(const float* w4) {
+    return __fadd_rn(__fadd_rn(w4[0], w4[1]), __fadd_rn(w4[2], w4[3]));
+}
+// silu(g) * u with silu(g) = g * 1 / (1 + 2^(-g log2 e)): ex2.approx, correctly rounded reciprocal
+__device__ __forceinline__ float swiglu_value(float g, float u) {
+    const float e = ex2_ftz(__fmul_rn(g, -LOG2E_F));
+    const float sig = __frcp_rn(__fadd_rn(1.0f, e));
+    return __fmul_rn(__fmul_rn(g, sig), u);
+}
+
 }  // namespace tik

@@ -96,4 +96,25 @@ struct LogprobParams {
 cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p,
                            cudaStream_t stream);
 
+struct NormParams {
+    const __nv_bfloat16* x;      // [T][H]
+    __nv_bfloat16* residual;     // [T][H] in/out, or null (plain RMSNorm)
+    const __nv_bfloat16* weight; // [H]
+    __nv_bfloat16* y;            // [T][H] (may be x)
+    float eps;
+    long long T;
+    int H;
+};
+cudaError_t launch_rmsnorm(const NormParams& p, cudaStream_t stream);
+cudaError_t launch_swiglu(const void* gate_up, void* out, long long T, int I, cudaStream_t stream);
+
+struct LinearParams {
+    __nv_bfloat16* y;            // [T][N]
+    int64_t T;
+    int K, N, nsuper;
+    int* dev_status;
+};
+cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const LinearParams& p,
+                          cudaStream_t stream);
+
 }  // namespace tik

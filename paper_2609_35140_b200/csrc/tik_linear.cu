@@ -1,0 +1,193 @@
+// Dense linear layer y = x W^T (bf16 in, fp32 accumulation in TMEM, bf16 out) for sm_100a: the
+// FFN projections of the unified operator set.  Same machinery as the log-probability GEMM: one
+// CTA = (128-row tile, 1024-column super-chunk); a TMA warp streams 64-wide K slices of x and W
+// through a four-stage shared-memory ring, an MMA warp accumulates the whole K range in ascending
+// order into one of two 256-column TMEM accumulators (M128 x N256 x K16, no split-K), and four
+// epilogue warps (one thread per row) round the accumulator to bf16 and store it while the next
+// 256 columns are being accumulated.  An output element is one fixed chain of MMAs over K, so it
+// depends on its x row and its W row only: a row gives the same bits whether it is computed alone
+// (decode) or inside a long batch (prefill, policy update).
+#include "tik_core.cuh"
+#include "tik_internal.h"
+#include "tik_ptx.cuh"
+
+namespace tik {
+
+namespace lin {
+constexpr int STAGES = 4;
+constexpr int NB = 256;                      // output columns per MMA
+constexpr int SUPER = 1024;                  // output columns per CTA
+constexpr uint32_t A_BYTES = 128 * 128;      // 128 rows x 64 bf16
+constexpr uint32_t B_BYTES = NB * 128;       // 256 W rows x 64 bf16
+constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t OFF_BAR = STAGES * STAGE_BYTES;
+constexpr uint32_t BYTES = OFF_BAR + 256;
+constexpr uint32_t ALLOC = BYTES + 1024;
+constexpr int BAND = 32;                     // row tiles per L2 band
+constexpr int THREADS = 192;                 // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+}  // namespace lin
+
+__global__ void __launch_bounds__(lin::THREADS, 1)
+linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+              const LinearParams p) {
+    using namespace lin;
+    constexpr uint32_t TMEM_COLS = 512;      // two 256-column accumulators
+    constexpr uint32_t IDESC = mma_idesc_bf16(128, NB, false);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // raster: bands of BAND row tiles; within a band the row tile varies fastest so the CTAs in
+    // flight share one super-chunk of W in L2 and W is streamed from HBM once per band
+    const int ntile = static_cast<int>((p.T + 127) / 128);
+    const long long per_band = static_cast<long long>(BAND) * p.nsuper;
+    const int band = static_cast<int>(blockIdx.x / per_band);
+    const int band_tiles = min(BAND, ntile - band * BAND);
+    const long long rem = blockIdx.x - band * per_band;
+    const int sup = static_cast<int>(rem / BAND);
+    const int tile_in_band = static_cast<int>(rem % BAND);
+    if (tile_in_band >= band_tiles) return;
+    const int row0 = (band * BAND + tile_in_band) * 128;
+    const int col_base = sup * SUPER;
+    const int n_nt = min(SUPER / NB, (p.N - col_base + NB - 1) / NB);   // 256-column steps
+    const int n_kb = p.K / 64;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t* smem = smem_raw + pad;
+    const uint32_t sbase = raw_addr + pad;
+    const uint32_t bar_full = sbase + OFF_BAR;               // STAGES barriers
+    const uint32_t bar_empty = bar_full + 8 * STAGES;        // STAGES barriers
+    const uint32_t bar_acc_full = bar_empty + 8 * STAGES;    // 2
+    const uint32_t bar_acc_empty = bar_acc_full + 16;        // 2
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 8 * (2 * STAGES + 4));
+    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + OFF_BAR + 8 * (2 * STAGES + 4) + 4);
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, 128);
+        }
+        *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int nt = 0; nt < n_nt; ++nt) {
+                const int col0 = col_base + nt * NB;
+                for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
+                    const int s = it % STAGES;
+                    const uint32_t use = it / STAGES;
+                    if (use > 0) mbar_wait(bar_empty + 8 * s, (use - 1) & 1, abort_word, p.dev_status);
+                    mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
+                    // rows past T and W rows past N are outside the tensor maps and arrive as zeros
+                    tma_load_2d(sbase + s * STAGE_BYTES, &tmA, bar_full + 8 * s, kb * 64, row0);
+                    tma_load_2d(sbase + s * STAGE_BYTES + A_BYTES, &tmB, bar_full + 8 * s, kb * 64, col0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int nt = 0; nt < n_nt; ++nt) {
+                const int buf = nt & 1;
+                const uint32_t use = nt >> 1;
+                if (use > 0) mbar_wait(bar_acc_empty + 8 * buf, (use - 1) & 1, abort_word, p.dev_status);
+                tc_fence_after();
+                for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    if (*abort_word) break;
+                    const int s = it % STAGES;
+                    mbar_wait(bar_full + 8 * s, (it / STAGES) & 1, abort_word, p.dev_status);
+                    tc_fence_after();
+                    const uint32_t a0 = sbase + s * STAGE_BYTES, b0 = a0 + A_BYTES;
+                    mma_ss_chain4(tmem + buf * NB, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
+                                  IDESC, kb ? 1u : 0u);
+                    mma_commit(bar_empty + 8 * s);
+                }
+                mma_commit(bar_acc_full + 8 * buf);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;                      // TMEM lane quarter of this warp
+        const int row = quarter * 32 + lane;
+        const long long t = static_cast<long long>(row0) + row;
+        const bool row_valid = t < p.T;
+        __nv_bfloat16* yrow = p.y + t * p.N;
+        for (int nt = 0; nt < n_nt; ++nt) {
+            const int buf = nt & 1;
+            mbar_wait(bar_acc_full + 8 * buf, (nt >> 1) & 1, abort_word, p.dev_status);
+            tc_fence_after();
+            const int col0 = col_base + nt * NB;
+            const uint32_t taddr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * NB;
+#pragma unroll 2
+            for (int cc = 0; cc < NB / 32; ++cc) {
+                if (col0 + 32 * cc >= p.N) break;              // warp-uniform: columns past N
+                uint32_t v[32];
+                tmem_ld32(taddr + 32 * cc, v);
+                tmem_wait_ld();
+                if (row_valid) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int col = col0 + 32 * cc + 8 * i;
+                        if (col < p.N)                         // N is a multiple of 8
+                            *reinterpret_cast<uint4*>(yrow + col) = make_uint4(
+                                pack_bf16x2(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
+                                pack_bf16x2(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
+                                pack_bf16x2(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
+                                pack_bf16x2(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
+                    }
+                }
+            }
+            // all TMEM reads of this accumulator are done: hand it back to the MMA warp
+            tc_fence_before();
+            mbar_arrive(bar_acc_empty + 8 * buf);
+        }
+    }
+
+    if (*abort_word) {   // let copies and MMAs in flight finish before shared memory and TMEM are released
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 1000000ull) {
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const LinearParams& p,
+                          cudaStream_t stream) {
+    if (p.T <= 0) return cudaSuccess;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(lin::ALLOC));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const long long ntile = (p.T + 127) / 128;
+    const long long nband = (ntile + lin::BAND - 1) / lin::BAND;
+    const long long grid = nband * lin::BAND * p.nsuper;
+    linear_kernel<<<static_cast<unsigned>(grid), lin::THREADS, lin::ALLOC, stream>>>(tmA, tmB, p);
+    return cudaGetLastError();
+}
+
+}  // namespace tik
