@@ -484,7 +484,14 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     p.T = T;
     p.K = K;
     p.N = N;
-    p.nsuper = (N + 1023) / 1024;
+    // Columns per CTA: 1024 amortises a CTA's set-up and lets the epilogue of one accumulator run
+    // under the MMAs of the next; with few row tiles (decode) that would leave SMs idle, so the
+    // super-chunk shrinks until the grid covers the SMs twice.  An output element is one
+    // 256-column accumulator's chain over K either way: its bits do not depend on this choice.
+    const long long ntile = (T + 127) / 128;
+    p.super_cols = 1024;
+    while (p.super_cols > 256 && ntile * ((N + p.super_cols - 1) / p.super_cols) < 2ll * ctx->sm_count) p.super_cols /= 2;
+    p.nsuper = (N + p.super_cols - 1) / p.super_cols;
     p.dev_status = ctx->dev_status;
     cudaError_t e = launch_linear(tmA, tmB, p, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_linear");

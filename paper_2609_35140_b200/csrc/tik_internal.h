@@ -112,6 +112,7 @@ struct LinearParams {
     __nv_bfloat16* y;            // [T][N]
     int64_t T;
     int K, N, nsuper;
+    int super_cols;              // output columns per CTA: 256, 512 or 1024
     int* dev_status;
 };
 cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const LinearParams& p,

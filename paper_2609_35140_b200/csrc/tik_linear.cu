@@ -1,6 +1,6 @@
 // Dense linear layer y = x W^T (bf16 in, fp32 accumulation in TMEM, bf16 out) for sm_100a: the
 // FFN projections of the unified operator set.  Same machinery as the log-probability GEMM: one
-// CTA = (128-row tile, 1024-column super-chunk); a TMA warp streams 64-wide K slices of x and W
+// CTA = (128-row tile, super-chunk of 256 to 1024 output columns); a TMA warp streams 64-wide K slices of x and W
 // through a four-stage shared-memory ring, an MMA warp accumulates the whole K range in ascending
 // order into one of two 256-column TMEM accumulators (M128 x N256 x K16, no split-K), and four
 // epilogue warps (one thread per row) round the accumulator to bf16 and store it while the next
@@ -16,7 +16,7 @@ namespace tik {
 namespace lin {
 constexpr int STAGES = 4;
 constexpr int NB = 256;                      // output columns per MMA
-constexpr int SUPER = 1024;                  // output columns per CTA
+constexpr int SUPER_MAX = 1024;              // output columns per CTA (256, 512 or 1024, chosen per launch)
 constexpr uint32_t A_BYTES = 128 * 128;      // 128 rows x 64 bf16
 constexpr uint32_t B_BYTES = NB * 128;       // 256 W rows x 64 bf16
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
@@ -46,8 +46,8 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const int tile_in_band = static_cast<int>(rem % BAND);
     if (tile_in_band >= band_tiles) return;
     const int row0 = (band * BAND + tile_in_band) * 128;
-    const int col_base = sup * SUPER;
-    const int n_nt = min(SUPER / NB, (p.N - col_base + NB - 1) / NB);   // 256-column steps
+    const int col_base = sup * p.super_cols;
+    const int n_nt = min(p.super_cols / NB, (p.N - col_base + NB - 1) / NB);   // 256-column steps
     const int n_kb = p.K / 64;
 
     extern __shared__ uint8_t smem_raw[];
