@@ -311,6 +311,61 @@ def time_prep(hp: "HotPath", reps: int = 5):
     return times[len(times) // 2], byt
 
 
+FFN_INTERMEDIATE = {256: 704, 1536: 8960, 3584: 18944, 4096: 12288, 5120: 27648}   # Qwen2.5 / Qwen3 class shapes
+
+
+def time_ffn(hp: "HotPath", peaks, tpeak, reps: int = 5):
+    """The FFN-side operators (hidden RMSNorm, fused residual + RMSNorm, gate/up projection, SwiGLU,
+    down projection) on up to 32 768 tokens of the workload's hidden size, each timed on its own
+    with an L2 flush before every launch.  Reported beside the step, not part of the metric."""
+    tik, w = hp.tik, hp.w
+    T, H = min(w.total_tokens, 32768), w.hidden
+    I = FFN_INTERMEDIATE.get(H, 4 * H)
+    gen = torch.Generator(device="cuda").manual_seed(w.seed + 4242)
+
+    def rn(shape, std=1.0):
+        return (torch.randn(shape, generator=gen, device="cuda") * std).to(torch.bfloat16)
+
+    x, res, wn = rn((T, H)), rn((T, H)), (1 + 0.1 * rn((H,)).float()).to(torch.bfloat16)
+    w_gu, w_d = rn((2 * I, H), 0.02), rn((H, I), 0.02)
+    h = torch.empty_like(x)
+    gu = torch.empty(T, 2 * I, dtype=torch.bfloat16, device="cuda")
+    act = torch.empty(T, I, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty_like(x)
+
+    def med(fn):
+        ts = []
+        for _ in range(reps + 2):
+            hp.flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        ts = sorted(ts[2:])
+        return ts[len(ts) // 2]
+
+    def hbm(ms, byt, note):
+        g = byt / (ms * 1e-3) / 1e9
+        return {"bound": "hbm", "achieved": g, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": g / peaks["hbm_gbs"],
+                "ms": ms, "bytes": byt, "note": note}
+
+    def tensor(ms, flops, note):
+        tf = flops / (ms * 1e-3) / 1e12
+        return {"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak, "ms": ms,
+                "note": note}
+
+    shape = "T=%d H=%d I=%d; beside the step, not part of the metric" % (T, H, I)
+    r = {}
+    r["rmsnorm"] = hbm(med(lambda: tik.tik_rmsnorm(x, wn, 1e-6, y=h)), 2 * T * H * 2, shape)
+    r["add_rmsnorm"] = hbm(med(lambda: tik.tik_rmsnorm(x, wn, 1e-6, residual=res, y=h)), 4 * T * H * 2, shape)
+    r["linear_gate_up"] = tensor(med(lambda: tik.tik_linear(h, w_gu, y=gu)), 2.0 * T * H * 2 * I, shape)
+    r["swiglu"] = hbm(med(lambda: tik.tik_swiglu(gu, out=act)), 3 * T * I * 2, shape)
+    r["linear_down"] = tensor(med(lambda: tik.tik_linear(act, w_d, y=out)), 2.0 * T * I * H, shape)
+    return r
+
+
 # ------------------------------------------------------------------------------------------
 def oracle_sample_ms(w: synth.Workload, budget_rows: int = 0, seed: int = 0):
     """Times the CPU oracle on a bounded sample of the workload's attention rows and scales
@@ -484,6 +539,7 @@ def main():
             "bound": "hbm", "achieved": g, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": g / peaks["hbm_gbs"],
             "ms": t_prep, "bytes": b_prep,
             "note": "pre-attention step over all tokens of the workload; measured after the timed steps, not part of the metric"}
+        rooflines.update(time_ffn(hp, peaks, burst))    # timed alone: held against the burst peak
         flags |= tik.device_status()
 
     cpu = None
