@@ -225,3 +225,20 @@ def linear(x, W, f32: bool = False):
     rc = getattr(lib(), "oracle_linear" + sfx)(_p(x), _p(W), ctypes.c_int64(T), ctypes.c_int(K), ctypes.c_int(N), _p(y))
     assert rc == 0
     return y
+
+
+def attn_bwd_packed(q, k, v, dout, cu_seqlens, scale: float, f32: bool = False):
+    """Backward of attn_packed: q, dout [tot,Hq,d], k, v [tot,Hkv,d] -> (dq, dk, dv)."""
+    q, k, v, dout, cu = _f32(q), _f32(k), _f32(v), _f32(dout), _i32(cu_seqlens)
+    tot, Hq, d = q.shape
+    Hkv = k.shape[1]
+    assert dout.shape == q.shape and v.shape == k.shape and cu[-1] == tot
+    dt, sfx = _real(f32)
+    dq = np.empty((tot, Hq, d), dtype=dt)
+    dk = np.empty((tot, Hkv, d), dtype=dt)
+    dv = np.empty((tot, Hkv, d), dtype=dt)
+    rc = getattr(lib(), "oracle_attn_bwd_packed" + sfx)(
+        _p(q), _p(k), _p(v), _p(dout), _p(cu), ctypes.c_int(len(cu) - 1), ctypes.c_int(Hq), ctypes.c_int(Hkv),
+        ctypes.c_int(d), ctypes.c_double(scale), _p(dq), _p(dk), _p(dv))
+    assert rc == 0
+    return dq, dk, dv
