@@ -53,6 +53,7 @@ typedef int tik_status;
 #define TIK_OP_ATTN_PREFILL 1
 #define TIK_OP_ATTN_DECODE 2
 #define TIK_OP_TOKEN_LOGPROB 3
+#define TIK_OP_ATTN_TRAIN_BWD 4
 
 /* Create / destroy the per-device context (host memory plus one small device status
  * word).  `device` is a CUDA ordinal.  tik_create is the only call that allocates. */
@@ -86,6 +87,22 @@ tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const 
                               float* lse, const int32_t* cu_seqlens, int S,
                               int64_t total_tokens, int max_seqlen, int Hq, int Hkv, int d,
                               float softmax_scale, void* stream);
+
+/* Backward of tik_attn_train_fwd (the paper measures the policy-update backward in its layer
+ * timings, Sec. 6 Q2, and does not put it under Eq. 1: there is no rollout counterpart).  Given
+ * dO = dL/dO it returns dQ, dK, dV of the same shapes as q, k, v (bf16, one rounding of fp32
+ * accumulators).  With s_ij = scale q_i.k_j, p_ij = exp(s_ij - lse_i), delta_i = dO_i.o_i:
+ *   dS_ij = p_ij (dO_i.v_j - delta_i),  dQ_i = scale sum_j dS_ij k_j,
+ *   dK_j = scale sum_i dS_ij q_i,  dV_j = sum_i p_ij dO_i      (sums over the query heads of a KV head too)
+ * o and lse are the forward's outputs for the same q, k, v, scale (lse: fp32 [total_tokens][Hq]).
+ * Deterministic: every output element is accumulated in one fixed order (no atomics); the same
+ * inputs give the same bits on every call.  ws: tik_workspace_bytes(TIK_OP_ATTN_TRAIN_BWD,
+ * total_tokens, Hq, ...) bytes of device scratch.  Three kernels on `stream`. */
+tik_status tik_attn_train_bwd(tik_ctx* ctx, const void* q, const void* k, const void* v, const void* o,
+                              const void* d_o, const float* lse, void* dq, void* dk, void* dv,
+                              const int32_t* cu_seqlens, int S, int64_t total_tokens, int max_seqlen,
+                              int Hq, int Hkv, int d, float softmax_scale, void* ws, size_t ws_bytes,
+                              void* stream);
 
 /* Indexed KV-cache write (paper Sec. 4.1: a rollout-only operator; exact copy).  The new
  * tokens of sequence s are rows cu_seqlens_new[s] .. cu_seqlens_new[s+1]-1 of k_new/v_new

@@ -16,7 +16,7 @@ import torch
 from . import build as _build
 
 OK = 0
-OP_ATTN_TRAIN_FWD, OP_ATTN_PREFILL, OP_ATTN_DECODE, OP_TOKEN_LOGPROB = 0, 1, 2, 3
+OP_ATTN_TRAIN_FWD, OP_ATTN_PREFILL, OP_ATTN_DECODE, OP_TOKEN_LOGPROB, OP_ATTN_TRAIN_BWD = 0, 1, 2, 3, 4
 DEV_BAD_BLOCK, DEV_BAD_TARGET, DEV_WAIT_EXPIRED, DEV_BAD_POSITION = 1, 2, 4, 8
 
 _lib = None
@@ -62,13 +62,16 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.tik_rmsnorm.argtypes = [vp, vp, vp, vp, vp, f32, i64, i32, vp]
     lib.tik_swiglu.argtypes = [vp, vp, vp, i64, i32, vp]
     lib.tik_linear.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp]
+    lib.tik_attn_train_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32,
+                                       vp, sz, vp]
     lib.tik_token_logprob.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, f32, vp, sz, vp]
     lib.tik_attn_decode_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
                                            i32, f32, vp, vp]
     lib.tik_attn_decode_static.restype = i32
     for name in ("tik_create", "tik_destroy", "tik_device_status", "tik_attn_train_fwd",
                  "tik_kv_cache_write", "tik_attn_prefill", "tik_attn_decode", "tik_token_logprob",
-                 "tik_qk_norm_rope_kv_write", "tik_rmsnorm", "tik_swiglu", "tik_linear"):
+                 "tik_qk_norm_rope_kv_write", "tik_rmsnorm", "tik_swiglu", "tik_linear",
+                 "tik_attn_train_bwd"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -141,6 +144,25 @@ def tik_attn_train_fwd(q, k, v, cu_seqlens, max_seqlen: int, softmax_scale: floa
                                    softmax_scale, _stream())
     _check(rc, ctx)
     return o
+
+
+def tik_attn_train_bwd(q, k, v, o, d_o, lse, cu_seqlens, max_seqlen: int, softmax_scale: float,
+                       ws: Optional[torch.Tensor] = None):
+    """Backward of tik_attn_train_fwd: returns (dq, dk, dv).  o, lse are the forward's outputs."""
+    ctx = context()
+    bf = torch.bfloat16
+    tot, Hq, d = q.shape
+    Hkv = k.shape[1]
+    need = workspace_bytes(OP_ATTN_TRAIN_BWD, tot, Hq, Hkv, d)
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    rc = load().tik_attn_train_bwd(ctx, _ptr(q, bf), _ptr(k, bf), _ptr(v, bf), _ptr(o, bf), _ptr(d_o, bf),
+                                   _ptr(lse, torch.float32), _ptr(dq, bf), _ptr(dk, bf), _ptr(dv, bf),
+                                   _ptr(cu_seqlens, torch.int32), cu_seqlens.numel() - 1, tot, max_seqlen, Hq, Hkv, d,
+                                   softmax_scale, _ptr(ws), ws.numel(), _stream())
+    _check(rc, ctx)
+    return dq, dk, dv
 
 
 def tik_kv_cache_write(k_new, v_new, cu_seqlens_new, ctx_lens, k_cache, v_cache, block_table):

@@ -137,6 +137,10 @@ size_t tik_workspace_bytes(int op, int64_t rows_or_batch, int Hq, int Hkv, int d
         const int64_t nsuper = (V + LP_SUPER - 1) / LP_SUPER;
         return static_cast<size_t>(rows_or_batch) * (2 * nsuper + 1) * sizeof(float);
     }
+    if (op == TIK_OP_ATTN_TRAIN_BWD) {      // rows_or_batch = total tokens: delta [tokens][Hq]
+        if (rows_or_batch <= 0) return 0;
+        return static_cast<size_t>(rows_or_batch) * Hq * sizeof(float);
+    }
     return 0;
 }
 
@@ -495,6 +499,54 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     p.dev_status = ctx->dev_status;
     cudaError_t e = launch_linear(tmA, tmB, p, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_linear");
+}
+
+tik_status tik_attn_train_bwd(tik_ctx* ctx, const void* q, const void* k, const void* v, const void* o,
+                              const void* d_o, const float* lse, void* dq, void* dk, void* dv,
+                              const int32_t* cu_seqlens, int S, int64_t total_tokens, int max_seqlen, int Hq,
+                              int Hkv, int d, float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    if (S < 0 || total_tokens < 0 || max_seqlen < 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative size");
+    tik_status st = check_heads(ctx, Hq, Hkv, d, softmax_scale);
+    if (st != TIK_OK) return st;
+    if (S == 0 || total_tokens == 0 || max_seqlen == 0) return TIK_OK;
+    if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv || !cu_seqlens)
+        return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
+        return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (total_tokens >= (1ll << 31)) return fail(ctx, TIK_ERR_UNSUPPORTED, "total_tokens must be < 2^31");
+    const size_t need = tik_workspace_bytes(TIK_OP_ATTN_TRAIN_BWD, total_tokens, Hq, Hkv, d, 0, 0, 0);
+    if (!ws || ws_bytes < need) return fail(ctx, TIK_ERR_WORKSPACE, "backward workspace too small");
+    if (S > 65535 || Hq > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "S and Hq must be <= 65535");
+
+    CUtensorMap tmQ, tmK, tmV, tmDO;
+    std::string err;
+    const uint64_t ud = static_cast<uint64_t>(d);
+    uint64_t qd[3] = {ud, static_cast<uint64_t>(Hq), static_cast<uint64_t>(total_tokens)};
+    uint64_t qs[2] = {ud * 2, ud * 2 * Hq};
+    uint64_t kd[3] = {ud, static_cast<uint64_t>(Hkv), static_cast<uint64_t>(total_tokens)};
+    uint64_t ks[2] = {ud * 2, ud * 2 * Hkv};
+    uint32_t box[3] = {64, 1, 128};
+    if (!make_tmap_bf16(ctx, &tmQ, q, 3, qd, qs, box, &err) || !make_tmap_bf16(ctx, &tmDO, d_o, 3, qd, qs, box, &err) ||
+        !make_tmap_bf16(ctx, &tmK, k, 3, kd, ks, box, &err) || !make_tmap_bf16(ctx, &tmV, v, 3, kd, ks, box, &err))
+        return fail(ctx, TIK_ERR_CUDA, err.c_str());
+    BwdParams p{};
+    p.cu_seqlens = cu_seqlens;
+    p.lse = lse;
+    p.delta = static_cast<float*>(ws);
+    p.dq = static_cast<__nv_bfloat16*>(dq);
+    p.dk = static_cast<__nv_bfloat16*>(dk);
+    p.dv = static_cast<__nv_bfloat16*>(dv);
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.G = Hq / Hkv;
+    p.c = scale_to_c(softmax_scale);
+    p.scale = softmax_scale;
+    p.dev_status = ctx->dev_status;
+    cudaError_t e = launch_attn_bwd(d, (max_seqlen + 127) / 128, S, tmQ, tmK, tmV, tmDO, p, o, d_o,
+                                    total_tokens * Hq, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_train_bwd");
 }
 
 }  // extern "C"

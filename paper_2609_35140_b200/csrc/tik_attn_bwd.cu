@@ -1,0 +1,378 @@
+// Backward of the packed causal GQA attention (policy-update backward) for sm_100a.
+//
+// Deterministic by construction: no atomics and no split accumulation.  Two launches of one
+// kernel body recompute the score tiles and differ in which side stays resident:
+//   DQ  mode: a CTA owns one 128-row query tile of one (sequence, head) and walks the KV tiles
+//             0..i:      S = Q_i K_j^T, dP = dO_i V_j^T, dS = P o (dP - delta) * scale,
+//             dQ_i += dS K_j                                     (accumulator in TMEM)
+//   DKV mode: a CTA owns one 128-row KV tile of one (sequence, KV head) and walks the query
+//             tiles i >= j of the G query heads of that KV head, one after the other:
+//             S^T = K_j Q_i^T, dP^T = V_j dO_i^T, dV_j += P^T dO_i, dK_j += dS^T Q_i
+// with P = exp2(S c - lse log2 e) from the forward's log-sum-exp and delta = rowsum(dO o O)
+// (a small kernel of its own).  All five products run on tcgen05: the two score products with
+// both operands in shared memory (TMA, 128B swizzle), the gradient products with the bf16
+// weights P / dS read from TMEM, written there in place of the fp32 scores they came from.
+// One TMA warp, one MMA-issuing warp, four element-wise warps (one thread per tile row).
+// Every wait is bounded and raises TIK_DEV_WAIT_EXPIRED instead of hanging.
+#include "tik_core.cuh"
+#include "tik_internal.h"
+#include "tik_ptx.cuh"
+
+namespace tik {
+
+enum { BWD_DQ = 0, BWD_DKV = 1 };
+constexpr int BWD_THREADS = 192;     // warp 0 TMA, warp 1 MMA, warps 2-5 element-wise
+constexpr int BWD_STAGES = 2;
+
+template <int D>
+struct BwdSmem {
+    static constexpr uint32_t ATOM = 128 * 128;           // 128 rows x 64 bf16
+    static constexpr uint32_t TILE = (D / 64) * ATOM;
+    static constexpr uint32_t OFF_R = 0;                  // two resident row-side tiles
+    static constexpr uint32_t OFF_C = 2 * TILE;           // BWD_STAGES x two streamed tiles
+    static constexpr uint32_t OFF_BAR = OFF_C + BWD_STAGES * 2 * TILE;
+    static constexpr uint32_t OFF_SC = OFF_BAR + 128;     // [2][2][128] floats: lse*log2e, delta of the columns
+    static constexpr uint32_t BYTES = OFF_SC + 2 * 2 * 128 * 4;
+    static constexpr uint32_t ALLOC = BYTES + 1024;       // slack to align the base to 1 KiB
+};
+
+template <int D, int MODE>
+__global__ void __launch_bounds__(BWD_THREADS, 1)
+attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
+                const BwdParams p) {
+    using L = BwdSmem<D>;
+    constexpr int NATOM = D / 64;
+    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t COL_T1 = 0, COL_T2 = 128, COL_A1 = 256, COL_A2 = 256 + D;
+    constexpr uint32_t IDESC_SC = mma_idesc_bf16(128, 128, false);
+    constexpr uint32_t IDESC_OUT = mma_idesc_bf16(128, D, true);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // ---------------------------------------------------------------- work item
+    const int seq = blockIdx.z;
+    const int tok0 = p.cu_seqlens[seq];
+    const int len = p.cu_seqlens[seq + 1] - tok0;
+    if (len <= 0) return;
+    const int nq = (len + 127) / 128;                      // tiles of the sequence (query and KV alike)
+    int own, head = 0, kvh, n_steps;
+    if (MODE == BWD_DQ) {
+        own = gridDim.x - 1 - blockIdx.x;                  // query tile, heaviest first
+        if (own >= nq) return;
+        head = blockIdx.y;
+        kvh = head / p.G;
+        n_steps = own + 1;                                 // KV tiles 0..own
+    } else {
+        own = blockIdx.x;                                  // KV tile, heaviest first
+        if (own >= nq) return;
+        kvh = blockIdx.y;
+        n_steps = p.G * (nq - own);                        // (g, query tile i >= own), g outermost
+    }
+    // step t -> the streamed tile and (DKV) the query head
+    auto step_tile = [&](int t) { return MODE == BWD_DQ ? t : own + t % (nq - own); };
+    auto step_head = [&](int t) { return MODE == BWD_DQ ? head : kvh * p.G + t / (nq - own); };
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t* smem = smem_raw + pad;
+    const uint32_t sbase = raw_addr + pad;
+    const uint32_t sR1 = sbase + L::OFF_R, sR2 = sR1 + L::TILE;
+    const uint32_t bar0 = sbase + L::OFF_BAR;
+    const uint32_t bar_r = bar0;                 // row-side tiles landed
+    const uint32_t bar_cfull = bar0 + 8;         // [2] streamed tiles landed
+    const uint32_t bar_cempty = bar0 + 24;       // [2] gradient MMAs that read the stage are done
+    const uint32_t bar_tfull = bar0 + 40;        // score MMAs of a step done
+    const uint32_t bar_efull = bar0 + 48;        // weights of a step written to TMEM (4 warps)
+    const uint32_t bar_acc = bar0 + 56;          // all MMAs done
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 64);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 68);
+    float* sc_l2 = reinterpret_cast<float*>(smem + L::OFF_SC);          // [2][128]
+    float* sc_dl = sc_l2 + 2 * 128;                                      // [2][128]
+
+    if (tid == 0) {
+        mbar_init(bar_r, 1);
+        for (int i = 0; i < BWD_STAGES; ++i) {
+            mbar_init(bar_cfull + 8 * i, 1);
+            mbar_init(bar_cempty + 8 * i, 1);
+        }
+        mbar_init(bar_tfull, 1);
+        mbar_init(bar_efull, 4);
+        mbar_init(bar_acc, 1);
+        *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmQ);
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
+        tma_prefetch_desc(&tmDO);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const int row_own = tok0 + 128 * own;
+            mbar_expect_tx(bar_r, 2 * L::TILE);
+            for (int a = 0; a < NATOM; ++a) {
+                if (MODE == BWD_DQ) {
+                    tma_load_3d(sR1 + a * L::ATOM, &tmQ, bar_r, a * 64, head, row_own);
+                    tma_load_3d(sR2 + a * L::ATOM, &tmDO, bar_r, a * 64, head, row_own);
+                } else {
+                    tma_load_3d(sR1 + a * L::ATOM, &tmK, bar_r, a * 64, kvh, row_own);
+                    tma_load_3d(sR2 + a * L::ATOM, &tmV, bar_r, a * 64, kvh, row_own);
+                }
+            }
+            for (int t = 0; t < n_steps; ++t) {
+                if (*abort_word) break;          // a wait expired somewhere: stop issuing copies
+                const int st = t % BWD_STAGES;
+                const uint32_t use = t / BWD_STAGES;
+                if (use > 0) mbar_wait(bar_cempty + 8 * st, (use - 1) & 1, abort_word, p.dev_status);
+                const uint32_t c1 = sbase + L::OFF_C + st * 2 * L::TILE, c2 = c1 + L::TILE;
+                const uint32_t full = bar_cfull + 8 * st;
+                const int row = tok0 + 128 * step_tile(t);
+                const int h = step_head(t);
+                mbar_expect_tx(full, 2 * L::TILE);
+                for (int a = 0; a < NATOM; ++a) {
+                    if (MODE == BWD_DQ) {
+                        tma_load_3d(c1 + a * L::ATOM, &tmK, full, a * 64, kvh, row);
+                        tma_load_3d(c2 + a * L::ATOM, &tmV, full, a * 64, kvh, row);
+                    } else {
+                        tma_load_3d(c1 + a * L::ATOM, &tmQ, full, a * 64, h, row);
+                        tma_load_3d(c2 + a * L::ATOM, &tmDO, full, a * 64, h, row);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        // MMAs issued by one thread execute in order: the score MMAs of step t+1 overwrite the
+        // columns that hold the weights of step t only after the gradient MMAs that read them.
+        if (lane == 0) {
+            mbar_wait(bar_r, 0, abort_word, p.dev_status);
+            const uint64_t dr1 = smem_desc_sw128(sR1, 0, 1024), dr2 = smem_desc_sw128(sR2, 0, 1024);
+            for (int t = 0; t < n_steps; ++t) {
+                if (*abort_word) break;
+                const int st = t % BWD_STAGES;
+                const uint32_t c1 = sbase + L::OFF_C + st * 2 * L::TILE, c2 = c1 + L::TILE;
+                mbar_wait(bar_cfull + 8 * st, (t / BWD_STAGES) & 1, abort_word, p.dev_status);
+                tc_fence_after();
+                if (D == 128) {
+                    mma_ss_chain8_fresh(tmem + COL_T1, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC);
+                    mma_ss_chain8_fresh(tmem + COL_T2, dr2, smem_desc_sw128(c2, 0, 1024), IDESC_SC);
+                } else {
+                    mma_ss_chain4_fresh(tmem + COL_T1, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC);
+                    mma_ss_chain4_fresh(tmem + COL_T2, dr2, smem_desc_sw128(c2, 0, 1024), IDESC_SC);
+                }
+                mma_commit(bar_tfull);
+                mbar_wait(bar_efull, t & 1, abort_word, p.dev_status);
+                tc_fence_after();
+                // gradient products: A = bf16 weights in TMEM, B = streamed tile (rows = contraction)
+                mma_ts_chain8(tmem + COL_A1, tmem + COL_T2, smem_desc_sw128(c1, L::ATOM, 1024), IDESC_OUT,
+                              t ? 1u : 0u);
+                if (MODE == BWD_DKV)
+                    mma_ts_chain8(tmem + COL_A2, tmem + COL_T1, smem_desc_sw128(c2, L::ATOM, 1024), IDESC_OUT,
+                                  t ? 1u : 0u);
+                mma_commit(bar_cempty + 8 * st);
+            }
+            mma_commit(bar_acc);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ element-wise warps
+        const int quarter = warp & 3;                      // TMEM lane quarter of this warp
+        const int r = quarter * 32 + lane;                 // tile row == TMEM lane
+        const int et = (warp - 2) * 32 + lane;             // 0..127 among the element-wise threads
+        const uint32_t tlane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+        const int row_abs = 128 * own + r;                 // position of this row in the sequence
+        const float c = p.c;                               // scale * log2(e)
+        float row_l2 = 0.0f, row_dl = 0.0f;
+        if (MODE == BWD_DQ && row_abs < len) {
+            const long long idx = (static_cast<long long>(tok0) + row_abs) * p.Hq + head;
+            row_l2 = __fmul_rn(p.lse[idx], LOG2E_F);
+            row_dl = p.delta[idx];
+        }
+        // DKV: the scalars belong to the columns (query rows of the streamed tile): element-wise
+        // thread `et` fetches those of column `et` one step ahead and passes them through shared memory
+        auto fetch_col = [&](int t, float& l2, float& dl) {
+            l2 = 0.0f;
+            dl = 0.0f;
+            if (t < n_steps) {
+                const int qa = 128 * step_tile(t) + et;
+                if (qa < len) {
+                    const long long idx = (static_cast<long long>(tok0) + qa) * p.Hq + step_head(t);
+                    l2 = __fmul_rn(p.lse[idx], LOG2E_F);
+                    dl = p.delta[idx];
+                }
+            }
+        };
+        if (MODE == BWD_DKV) {
+            float l2, dl;
+            fetch_col(0, l2, dl);
+            sc_l2[et] = l2;
+            sc_dl[et] = dl;
+            named_bar_sync(1, 128);
+        }
+        for (int t = 0; t < n_steps; ++t) {
+            float nl2 = 0.0f, ndl = 0.0f;
+            if (MODE == BWD_DKV) fetch_col(t + 1, nl2, ndl);          // in flight during this step
+            const int ct = step_tile(t);
+            const float* cl2 = sc_l2 + (t & 1) * 128;
+            const float* cdl = sc_dl + (t & 1) * 128;
+            mbar_wait(bar_tfull, t & 1, abort_word, p.dev_status);
+            tc_fence_after();
+            // column c of the tile is masked for this row when it lies in the row's future (DQ: key
+            // after query; DKV: query before key) or, DKV, past the end of the sequence
+            const int col0_abs = 128 * ct;
+#pragma unroll 1
+            for (int hlf = 0; hlf < 2; ++hlf) {
+                uint32_t s_[64], d_[64];
+                tmem_ld32(tlane + COL_T1 + 64 * hlf, *reinterpret_cast<uint32_t(*)[32]>(&s_[0]));
+                tmem_ld32(tlane + COL_T1 + 64 * hlf + 32, *reinterpret_cast<uint32_t(*)[32]>(&s_[32]));
+                tmem_ld32(tlane + COL_T2 + 64 * hlf, *reinterpret_cast<uint32_t(*)[32]>(&d_[0]));
+                tmem_ld32(tlane + COL_T2 + 64 * hlf + 32, *reinterpret_cast<uint32_t(*)[32]>(&d_[32]));
+                tmem_wait_ld();
+                uint32_t pk[32], dk_[32];
+#pragma unroll
+                for (int i = 0; i < 64; i += 2) {
+                    float pv[2], dsv[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int cc = 64 * hlf + i + e;
+                        const int col_abs = col0_abs + cc;
+                        bool masked;
+                        float l2, dl;
+                        if (MODE == BWD_DQ) {
+                            masked = col_abs > row_abs;
+                            l2 = row_l2;
+                            dl = row_dl;
+                        } else {
+                            masked = (row_abs > col_abs) || (col_abs >= len);
+                            l2 = cl2[cc];
+                            dl = cdl[cc];
+                        }
+                        const float pe = bwd_p(__uint_as_float(s_[i + e]), c, l2);
+                        pv[e] = masked ? 0.0f : pe;
+                        dsv[e] = masked ? 0.0f : bwd_ds(pe, __uint_as_float(d_[i + e]), dl, p.scale);
+                    }
+                    pk[i >> 1] = pack_bf16x2(pv[0], pv[1]);
+                    dk_[i >> 1] = pack_bf16x2(dsv[0], dsv[1]);
+                }
+                // in place: the 32 columns written here were read in this or the previous half
+                if (MODE == BWD_DKV) tmem_st32(tlane + COL_T1 + 32 * hlf, pk);
+                tmem_st32(tlane + COL_T2 + 32 * hlf, dk_);
+            }
+            tmem_wait_st();
+            if (MODE == BWD_DKV) {
+                // hand the next step's column scalars over (the buffer was last read two steps ago)
+                sc_l2[((t + 1) & 1) * 128 + et] = nl2;
+                sc_dl[((t + 1) & 1) * 128 + et] = ndl;
+                named_bar_sync(1, 128);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_efull);
+        }
+        // ---- epilogue: fp32 accumulators -> bf16 rows
+        mbar_wait(bar_acc, 0, abort_word, p.dev_status);
+        tc_fence_after();
+        const bool valid = row_abs < len;
+        const long long tok = static_cast<long long>(tok0) + row_abs;
+        __nv_bfloat16* out1 = (MODE == BWD_DQ) ? p.dq + (tok * p.Hq + head) * D : p.dk + (tok * p.Hkv + kvh) * D;
+        __nv_bfloat16* out2 = p.dv + (tok * p.Hkv + kvh) * D;
+#pragma unroll 1
+        for (int which = 0; which < (MODE == BWD_DKV ? 2 : 1); ++which) {
+            const uint32_t col = which ? COL_A2 : COL_A1;
+            __nv_bfloat16* out = which ? out2 : out1;
+#pragma unroll
+            for (int cc = 0; cc < D / 32; ++cc) {
+                uint32_t v[32];
+                tmem_ld32(tlane + col + 32 * cc, v);
+                tmem_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        reinterpret_cast<uint4*>(out + 32 * cc)[i] = make_uint4(
+                            pack_bf16x2(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
+                            pack_bf16x2(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
+                            pack_bf16x2(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
+                            pack_bf16x2(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
+                }
+            }
+        }
+    }
+
+    if (*abort_word) {   // let copies and MMAs in flight finish before shared memory and TMEM are released
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 1000000ull) {
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// delta[token][head] = sum_c dO * O in fp32: one warp per (token, head), lane chain then butterfly.
+template <int D>
+__global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16* __restrict__ o,
+                                                       const __nv_bfloat16* __restrict__ dout,
+                                                       float* __restrict__ delta, long long n_vec) {
+    const long long v = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (v >= n_vec) return;
+    constexpr int EPL = D / 32;                             // elements per lane (4 or 2)
+    const __nv_bfloat16* op = o + v * D + EPL * lane;
+    const __nv_bfloat16* dp = dout + v * D + EPL * lane;
+    float part = 0.0f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) part = __fmaf_rn(__bfloat162float(dp[e]), __bfloat162float(op[e]), part);
+    part = hn_warp_total(part);
+    if (lane == 0) delta[v] = part;
+}
+
+template <int D, int MODE>
+static cudaError_t launch_bwd_t(dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                                const CUtensorMap& tmDO, const BwdParams& p, cudaStream_t stream) {
+    auto kern = attn_bwd_kernel<D, MODE>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(BwdSmem<D>::ALLOC));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    kern<<<grid, BWD_THREADS, BwdSmem<D>::ALLOC, stream>>>(tmQ, tmK, tmV, tmDO, p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_attn_bwd(int d, int max_tiles, int S, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                            const CUtensorMap& tmV, const CUtensorMap& tmDO, const BwdParams& p,
+                            const void* o, const void* dout, long long n_vec, cudaStream_t stream) {
+    const unsigned dgrid = static_cast<unsigned>((n_vec * 32 + 255) / 256);
+    if (d == 128)
+        bwd_delta_kernel<128><<<dgrid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(o),
+                                                         static_cast<const __nv_bfloat16*>(dout), p.delta, n_vec);
+    else
+        bwd_delta_kernel<64><<<dgrid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(o),
+                                                        static_cast<const __nv_bfloat16*>(dout), p.delta, n_vec);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const dim3 gq(max_tiles, p.Hq, S), gkv(max_tiles, p.Hkv, S);
+    if (d == 128) {
+        e = launch_bwd_t<128, BWD_DKV>(gkv, tmQ, tmK, tmV, tmDO, p, stream);
+        if (e == cudaSuccess) e = launch_bwd_t<128, BWD_DQ>(gq, tmQ, tmK, tmV, tmDO, p, stream);
+    } else {
+        e = launch_bwd_t<64, BWD_DKV>(gkv, tmQ, tmK, tmV, tmDO, p, stream);
+        if (e == cudaSuccess) e = launch_bwd_t<64, BWD_DQ>(gq, tmQ, tmK, tmV, tmDO, p, stream);
+    }
+    return e;
+}
+
+}  // namespace tik

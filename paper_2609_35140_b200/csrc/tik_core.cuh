@@ -241,4 +241,11 @@ __device__ __forceinline__ float swiglu_value(float g, float u) {
     return __fmul_rn(__fmul_rn(g, sig), u);
 }
 
+// ---- attention backward: weight and score gradient of one (query, key) pair ------------------
+// p = 2^(s c - lse log2 e) with the forward's log-sum-exp; ds = (p (dp - delta)) scale.
+__device__ __forceinline__ float bwd_p(float s, float c, float lse_log2) { return ex2_ftz(__fmaf_rn(s, c, -lse_log2)); }
+__device__ __forceinline__ float bwd_ds(float p, float dp, float delta, float scale) {
+    return __fmul_rn(__fmul_rn(p, __fsub_rn(dp, delta)), scale);
+}
+
 }  // namespace tik

@@ -118,4 +118,20 @@ struct LinearParams {
 cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const LinearParams& p,
                           cudaStream_t stream);
 
+struct BwdParams {
+    const int32_t* cu_seqlens;   // [S+1]
+    const float* lse;            // [total][Hq], natural log, from the forward
+    float* delta;                // [total][Hq] scratch: rowsum(dO o O)
+    __nv_bfloat16* dq;           // [total][Hq][d]
+    __nv_bfloat16* dk;           // [total][Hkv][d]
+    __nv_bfloat16* dv;           // [total][Hkv][d]
+    int Hq, Hkv, G;
+    float c;                     // softmax_scale * log2(e)
+    float scale;
+    int* dev_status;
+};
+cudaError_t launch_attn_bwd(int d, int max_tiles, int S, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                            const CUtensorMap& tmV, const CUtensorMap& tmDO, const BwdParams& p,
+                            const void* o, const void* dout, long long n_vec, cudaStream_t stream);
+
 }  // namespace tik
