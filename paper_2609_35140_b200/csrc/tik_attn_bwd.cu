@@ -12,7 +12,10 @@
 // (a small kernel of its own).  All five products run on tcgen05: the two score products with
 // both operands in shared memory (TMA, 128B swizzle), the gradient products with the bf16
 // weights P / dS read from TMEM, written there in place of the fp32 scores they came from.
-// One TMA warp, one MMA-issuing warp, four element-wise warps (one thread per tile row).
+// One TMA warp, one MMA-issuing warp, and two element-wise warpgroups (one thread per tile row
+// each).  A step's 128 streamed rows are handled as two halves of 64: warpgroup h turns the score
+// columns of half h into weights while the tensor pipe runs the gradient product of the other
+// half and the score product of the next step, so MMAs and element-wise work overlap.
 // Every wait is bounded and raises TIK_DEV_WAIT_EXPIRED instead of hanging.
 #include "tik_core.cuh"
 #include "tik_internal.h"
@@ -21,7 +24,7 @@
 namespace tik {
 
 enum { BWD_DQ = 0, BWD_DKV = 1 };
-constexpr int BWD_THREADS = 192;     // warp 0 TMA, warp 1 MMA, warps 2-5 element-wise
+constexpr int BWD_THREADS = 320;     // warp 0 TMA, warp 1 MMA, warps 2-9 element-wise (two per tile row)
 constexpr int BWD_STAGES = 2;
 
 template <int D>
@@ -31,8 +34,8 @@ struct BwdSmem {
     static constexpr uint32_t OFF_R = 0;                  // two resident row-side tiles
     static constexpr uint32_t OFF_C = 2 * TILE;           // BWD_STAGES x two streamed tiles
     static constexpr uint32_t OFF_BAR = OFF_C + BWD_STAGES * 2 * TILE;
-    static constexpr uint32_t OFF_SC = OFF_BAR + 128;     // [2][2][128] floats: lse*log2e, delta of the columns
-    static constexpr uint32_t BYTES = OFF_SC + 2 * 2 * 128 * 4;
+    static constexpr uint32_t OFF_SC = OFF_BAR + 128;     // [half][buffer][l2 | delta][64] floats of the columns
+    static constexpr uint32_t BYTES = OFF_SC + 2 * 2 * 2 * 64 * 4;
     static constexpr uint32_t ALLOC = BYTES + 1024;       // slack to align the base to 1 KiB
 };
 
@@ -45,7 +48,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     constexpr int NATOM = D / 64;
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t COL_T1 = 0, COL_T2 = 128, COL_A1 = 256, COL_A2 = 256 + D;
-    constexpr uint32_t IDESC_SC = mma_idesc_bf16(128, 128, false);
+    constexpr uint32_t IDESC_SC = mma_idesc_bf16(128, 64, false);       // one half: 64 streamed rows
     constexpr uint32_t IDESC_OUT = mma_idesc_bf16(128, D, true);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -82,13 +85,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t bar_r = bar0;                 // row-side tiles landed
     const uint32_t bar_cfull = bar0 + 8;         // [2] streamed tiles landed
     const uint32_t bar_cempty = bar0 + 24;       // [2] gradient MMAs that read the stage are done
-    const uint32_t bar_tfull = bar0 + 40;        // score MMAs of a step done
-    const uint32_t bar_efull = bar0 + 48;        // weights of a step written to TMEM (4 warps)
-    const uint32_t bar_acc = bar0 + 56;          // all MMAs done
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 64);
-    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 68);
-    float* sc_l2 = reinterpret_cast<float*>(smem + L::OFF_SC);          // [2][128]
-    float* sc_dl = sc_l2 + 2 * 128;                                      // [2][128]
+    const uint32_t bar_tfull = bar0 + 40;        // [2] score MMAs of a half-step done
+    const uint32_t bar_efull = bar0 + 56;        // [2] weights of a half-step written to TMEM (4 warps)
+    const uint32_t bar_acc = bar0 + 72;          // all MMAs done
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 80);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 84);
+    float* sc_base = reinterpret_cast<float*>(smem + L::OFF_SC);
 
     if (tid == 0) {
         mbar_init(bar_r, 1);
@@ -96,8 +98,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_init(bar_cfull + 8 * i, 1);
             mbar_init(bar_cempty + 8 * i, 1);
         }
-        mbar_init(bar_tfull, 1);
-        mbar_init(bar_efull, 4);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_tfull + 8 * i, 1);
+            mbar_init(bar_efull + 8 * i, 4);
+        }
         mbar_init(bar_acc, 1);
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
         fence_barrier_init();
@@ -153,34 +157,48 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        // MMAs issued by one thread execute in order: the score MMAs of step t+1 overwrite the
-        // columns that hold the weights of step t only after the gradient MMAs that read them.
+        // MMAs issued by one thread execute in order: the score MMAs of half h of step t+1 overwrite
+        // the columns that hold the weights of half h of step t only after the gradient MMAs that
+        // read them.  Issue order per step: gradient(a,t), score(a,t+1), gradient(b,t), score(b,t+1).
         if (lane == 0) {
             mbar_wait(bar_r, 0, abort_word, p.dev_status);
             const uint64_t dr1 = smem_desc_sw128(sR1, 0, 1024), dr2 = smem_desc_sw128(sR2, 0, 1024);
+            auto stage_c1 = [&](int t) { return sbase + L::OFF_C + (t % BWD_STAGES) * 2 * L::TILE; };
+            auto score = [&](int t, int h) {      // T1h = R1 C1h^T, T2h = R2 C2h^T (64 streamed rows = 8 KiB)
+                const uint32_t c1 = stage_c1(t) + h * 8192, c2 = c1 + L::TILE;
+                if (D == 128) {
+                    mma_ss_chain8_fresh(tmem + COL_T1 + 64 * h, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC);
+                    mma_ss_chain8_fresh(tmem + COL_T2 + 64 * h, dr2, smem_desc_sw128(c2, 0, 1024), IDESC_SC);
+                } else {
+                    mma_ss_chain4_fresh(tmem + COL_T1 + 64 * h, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC);
+                    mma_ss_chain4_fresh(tmem + COL_T2 + 64 * h, dr2, smem_desc_sw128(c2, 0, 1024), IDESC_SC);
+                }
+                mma_commit(bar_tfull + 8 * h);
+            };
+            auto gradient = [&](int t, int h) {   // A = bf16 weights of half h in TMEM, B = its 64 streamed rows
+                const uint32_t c1 = stage_c1(t) + h * 8192, c2 = c1 + L::TILE;
+                const uint32_t acc = (t > 0 || h > 0) ? 1u : 0u;
+                mma_ts_chain4(tmem + COL_A1, tmem + COL_T2 + 64 * h, smem_desc_sw128(c1, L::ATOM, 1024), IDESC_OUT, acc);
+                if (MODE == BWD_DKV)
+                    mma_ts_chain4(tmem + COL_A2, tmem + COL_T1 + 64 * h, smem_desc_sw128(c2, L::ATOM, 1024), IDESC_OUT,
+                                  acc);
+            };
+            mbar_wait(bar_cfull, 0, abort_word, p.dev_status);
+            tc_fence_after();
+            score(0, 0);
+            score(0, 1);
             for (int t = 0; t < n_steps; ++t) {
                 if (*abort_word) break;
-                const int st = t % BWD_STAGES;
-                const uint32_t c1 = sbase + L::OFF_C + st * 2 * L::TILE, c2 = c1 + L::TILE;
-                mbar_wait(bar_cfull + 8 * st, (t / BWD_STAGES) & 1, abort_word, p.dev_status);
-                tc_fence_after();
-                if (D == 128) {
-                    mma_ss_chain8_fresh(tmem + COL_T1, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC);
-                    mma_ss_chain8_fresh(tmem + COL_T2, dr2, smem_desc_sw128(c2, 0, 1024), IDESC_SC);
-                } else {
-                    mma_ss_chain4_fresh(tmem + COL_T1, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC);
-                    mma_ss_chain4_fresh(tmem + COL_T2, dr2, smem_desc_sw128(c2, 0, 1024), IDESC_SC);
+                const bool more = t + 1 < n_steps;
+                if (more) mbar_wait(bar_cfull + 8 * ((t + 1) % BWD_STAGES), ((t + 1) / BWD_STAGES) & 1, abort_word,
+                                    p.dev_status);
+                for (int h = 0; h < 2; ++h) {
+                    mbar_wait(bar_efull + 8 * h, t & 1, abort_word, p.dev_status);
+                    tc_fence_after();
+                    gradient(t, h);
+                    if (h == 1) mma_commit(bar_cempty + 8 * (t % BWD_STAGES));     // stage of step t consumed
+                    if (more) score(t + 1, h);
                 }
-                mma_commit(bar_tfull);
-                mbar_wait(bar_efull, t & 1, abort_word, p.dev_status);
-                tc_fence_after();
-                // gradient products: A = bf16 weights in TMEM, B = streamed tile (rows = contraction)
-                mma_ts_chain8(tmem + COL_A1, tmem + COL_T2, smem_desc_sw128(c1, L::ATOM, 1024), IDESC_OUT,
-                              t ? 1u : 0u);
-                if (MODE == BWD_DKV)
-                    mma_ts_chain8(tmem + COL_A2, tmem + COL_T1, smem_desc_sw128(c2, L::ATOM, 1024), IDESC_OUT,
-                                  t ? 1u : 0u);
-                mma_commit(bar_cempty + 8 * st);
             }
             mma_commit(bar_acc);
         }
@@ -189,7 +207,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // ------------------------------------------------------------ element-wise warps
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
         const int r = quarter * 32 + lane;                 // tile row == TMEM lane
-        const int et = (warp - 2) * 32 + lane;             // 0..127 among the element-wise threads
+        const int hlf = (warp - 2) >> 2;                   // which 64 columns of the row this thread owns
+        const int et = ((warp - 2) & 3) * 32 + lane;       // 0..127 within the thread's group of four warps
         const uint32_t tlane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const int row_abs = 128 * own + r;                 // position of this row in the sequence
         const float c = p.c;                               // scale * log2(e)
@@ -199,13 +218,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             row_l2 = __fmul_rn(p.lse[idx], LOG2E_F);
             row_dl = p.delta[idx];
         }
-        // DKV: the scalars belong to the columns (query rows of the streamed tile): element-wise
-        // thread `et` fetches those of column `et` one step ahead and passes them through shared memory
+        // DKV: the scalars belong to the columns (query rows of the streamed tile).  Thread `et` < 64
+        // of warpgroup h fetches those of column 64 h + et one step ahead; they reach the other
+        // threads of the warpgroup through shared memory (double-buffered, one named barrier per step).
+        float* my_sc = sc_base + hlf * (2 * 2 * 64);          // [buffer][64][l2, delta]
         auto fetch_col = [&](int t, float& l2, float& dl) {
             l2 = 0.0f;
             dl = 0.0f;
-            if (t < n_steps) {
-                const int qa = 128 * step_tile(t) + et;
+            if (t < n_steps && et < 64) {
+                const int qa = 128 * step_tile(t) + 64 * hlf + et;
                 if (qa < len) {
                     const long long idx = (static_cast<long long>(tok0) + qa) * p.Hq + step_head(t);
                     l2 = __fmul_rn(p.lse[idx], LOG2E_F);
@@ -216,23 +237,22 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (MODE == BWD_DKV) {
             float l2, dl;
             fetch_col(0, l2, dl);
-            sc_l2[et] = l2;
-            sc_dl[et] = dl;
-            named_bar_sync(1, 128);
+            if (et < 64) {
+                my_sc[2 * et] = l2;
+                my_sc[2 * et + 1] = dl;
+            }
+            named_bar_sync(1 + hlf, 128);
         }
         for (int t = 0; t < n_steps; ++t) {
             float nl2 = 0.0f, ndl = 0.0f;
-            if (MODE == BWD_DKV) fetch_col(t + 1, nl2, ndl);          // in flight during this step
-            const int ct = step_tile(t);
-            const float* cl2 = sc_l2 + (t & 1) * 128;
-            const float* cdl = sc_dl + (t & 1) * 128;
-            mbar_wait(bar_tfull, t & 1, abort_word, p.dev_status);
+            if (MODE == BWD_DKV) fetch_col(t + 1, nl2, ndl);            // in flight during this step
+            const float2* csc = reinterpret_cast<const float2*>(my_sc + (t & 1) * 128);   // (l2, delta) per column
+            mbar_wait(bar_tfull + 8 * hlf, t & 1, abort_word, p.dev_status);
             tc_fence_after();
-            // column c of the tile is masked for this row when it lies in the row's future (DQ: key
+            // column cc of the half is masked for this row when it lies in the row's future (DQ: key
             // after query; DKV: query before key) or, DKV, past the end of the sequence
-            const int col0_abs = 128 * ct;
-#pragma unroll 1
-            for (int hlf = 0; hlf < 2; ++hlf) {
+            const int col0_abs = 128 * step_tile(t) + 64 * hlf;
+            {
                 uint32_t s_[64], d_[64];
                 tmem_ld32(tlane + COL_T1 + 64 * hlf, *reinterpret_cast<uint32_t(*)[32]>(&s_[0]));
                 tmem_ld32(tlane + COL_T1 + 64 * hlf + 32, *reinterpret_cast<uint32_t(*)[32]>(&s_[32]));
@@ -245,7 +265,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     float pv[2], dsv[2];
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
-                        const int cc = 64 * hlf + i + e;
+                        const int cc = i + e;
                         const int col_abs = col0_abs + cc;
                         bool masked;
                         float l2, dl;
@@ -255,8 +275,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                             dl = row_dl;
                         } else {
                             masked = (row_abs > col_abs) || (col_abs >= len);
-                            l2 = cl2[cc];
-                            dl = cdl[cc];
+                            const float2 sc2 = csc[cc];
+                            l2 = sc2.x;
+                            dl = sc2.y;
                         }
                         const float pe = bwd_p(__uint_as_float(s_[i + e]), c, l2);
                         pv[e] = masked ? 0.0f : pe;
@@ -265,20 +286,23 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     pk[i >> 1] = pack_bf16x2(pv[0], pv[1]);
                     dk_[i >> 1] = pack_bf16x2(dsv[0], dsv[1]);
                 }
-                // in place: the 32 columns written here were read in this or the previous half
-                if (MODE == BWD_DKV) tmem_st32(tlane + COL_T1 + 32 * hlf, pk);
-                tmem_st32(tlane + COL_T2 + 32 * hlf, dk_);
+                // the weights go in place of the half's own scores (its first 32 columns)
+                if (MODE == BWD_DKV) tmem_st32(tlane + COL_T1 + 64 * hlf, pk);
+                tmem_st32(tlane + COL_T2 + 64 * hlf, dk_);
             }
             tmem_wait_st();
             if (MODE == BWD_DKV) {
-                // hand the next step's column scalars over (the buffer was last read two steps ago)
-                sc_l2[((t + 1) & 1) * 128 + et] = nl2;
-                sc_dl[((t + 1) & 1) * 128 + et] = ndl;
-                named_bar_sync(1, 128);
+                // hand the next step's column scalars over (the buffer was last read a step ago, before
+                // the previous barrier)
+                if (et < 64) {
+                    my_sc[((t + 1) & 1) * 128 + 2 * et] = nl2;
+                    my_sc[((t + 1) & 1) * 128 + 2 * et + 1] = ndl;
+                }
+                named_bar_sync(1 + hlf, 128);
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_efull);
+            if (lane == 0) mbar_arrive(bar_efull + 8 * hlf);
         }
         // ---- epilogue: fp32 accumulators -> bf16 rows
         mbar_wait(bar_acc, 0, abort_word, p.dev_status);
@@ -292,7 +316,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const uint32_t col = which ? COL_A2 : COL_A1;
             __nv_bfloat16* out = which ? out2 : out1;
 #pragma unroll
-            for (int cc = 0; cc < D / 32; ++cc) {
+            for (int cc = hlf * (D / 64); cc < (hlf + 1) * (D / 64); ++cc) {
                 uint32_t v[32];
                 tmem_ld32(tlane + col + 32 * cc, v);
                 tmem_wait_ld();

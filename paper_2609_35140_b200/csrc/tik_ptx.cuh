@@ -290,6 +290,18 @@ __device__ __forceinline__ void mma_ts_chain8(uint32_t d_tmem, uint32_t a_tmem, 
         : "memory");
 }
 
+// The first four of those steps (64 contraction rows).
+__device__ __forceinline__ void mma_ts_chain4(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                              uint32_t idesc, uint32_t first_accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p0, pt;\n\t.reg .b64 db;\n\t.reg .b32 ta;\n\t"
+        "setp.ne.b32 p0, %4, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+        TIK_MMA_TS_STEP(8, 128) TIK_MMA_TS_STEP(16, 256) TIK_MMA_TS_STEP(24, 384)
+        "}" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(first_accumulate)
+        : "memory");
+}
+
 // Arrives on the mbarrier once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
