@@ -311,6 +311,31 @@ def time_prep(hp: "HotPath", reps: int = 5):
     return times[len(times) // 2], byt
 
 
+def time_bwd(hp: "HotPath", burst, reps: int = 3):
+    """The policy-update backward of the train-forward phase (dQ, dK, dV), timed on its own."""
+    tik, w = hp.tik, hp.w
+    gen = torch.Generator(device="cuda").manual_seed(w.seed + 777)
+    do = torch.randn(hp.q.shape, generator=gen, device="cuda").to(torch.bfloat16)
+    lse = torch.empty(hp.q.shape[0], w.Hq, dtype=torch.float32, device="cuda")
+    o = tik.tik_attn_train_fwd(hp.q, hp.k, hp.v, hp.cu, max(w.seq_lens), w.softmax_scale, lse=lse)
+    ws = torch.empty(max(16, tik.workspace_bytes(tik.OP_ATTN_TRAIN_BWD, hp.q.shape[0], w.Hq, w.Hkv, w.d)),
+                     dtype=torch.uint8, device="cuda")
+    ts = []
+    for _ in range(reps + 1):
+        hp.flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        tik.tik_attn_train_bwd(hp.q, hp.k, hp.v, o, do, lse, hp.cu, max(w.seq_lens), w.softmax_scale, ws=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    ms = sorted(ts[1:])[len(ts[1:]) // 2]
+    tf = 2.5 * w.train_flops() / (ms * 1e-3) / 1e12
+    return {"bound": "tensor", "achieved": tf, "peak": burst, "unit": "TFLOP/s", "frac": tf / burst, "ms": ms,
+            "note": "algorithmic flops = 2.5 x the forward's (five products against two); the two-pass kernel "
+                    "executes 3.5 x; beside the step, not part of the metric"}
+
+
 FFN_INTERMEDIATE = {256: 704, 1536: 8960, 3584: 18944, 4096: 12288, 5120: 27648}   # Qwen2.5 / Qwen3 class shapes
 
 
@@ -540,6 +565,7 @@ def main():
             "ms": t_prep, "bytes": b_prep,
             "note": "pre-attention step over all tokens of the workload; measured after the timed steps, not part of the metric"}
         rooflines.update(time_ffn(hp, peaks, burst))    # timed alone: held against the burst peak
+        rooflines["attn_train_bwd"] = time_bwd(hp, burst)
         flags |= tik.device_status()
 
     cpu = None

@@ -123,3 +123,25 @@ def test_logprob_at_full_size(tik, index):
     for a, b in [(0, 1), (0, w.S), (T - 300, T), (1000, 1000 + 64)]:
         part = tik.tik_token_logprob(hidden[a:b].contiguous(), W, target[a:b].contiguous())
         assert count_diff(part, lp[a:b]) == 0, (a, b)
+
+
+def test_attention_backward_at_full_size(tik):
+    """Workload 1 at its real size; the oracle checks two whole sequences (sequences are independent)."""
+    w = synth.get_workload(1)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    do, _, _, _ = synth.make_qkv(w, "cuda", seed_offset=5)
+    lse = torch.empty(q.shape[0], w.Hq, dtype=torch.float32, device="cuda")
+    o = tik.tik_attn_train_fwd(q, k, v, cu, max(w.seq_lens), w.softmax_scale, lse=lse)
+    dq, dk, dv = tik.tik_attn_train_bwd(q, k, v, o, do, lse, cu, max(w.seq_lens), w.softmax_scale)
+    dq2, dk2, dv2 = tik.tik_attn_train_bwd(q, k, v, o, do, lse, cu, max(w.seq_lens), w.softmax_scale)
+    assert count_diff(dq, dq2) == 0 and count_diff(dk, dk2) == 0 and count_diff(dv, dv2) == 0
+    cu_h = w.cu_seqlens()
+    for s in (int(np.argmin(w.seq_lens)), int(np.argmax(w.seq_lens))):
+        sl = slice(int(cu_h[s]), int(cu_h[s + 1]))
+        rq, rk, rv = oracle.attn_bwd_packed(q[sl].float().cpu().numpy(), k[sl].float().cpu().numpy(),
+                                            v[sl].float().cpu().numpy(), do[sl].float().cpu().numpy(),
+                                            np.array([0, w.seq_lens[s]], dtype=np.int32), w.softmax_scale)
+        for got, ref in ((dq[sl], rq), (dk[sl], rk), (dv[sl], rv)):
+            err = got.float().cpu().numpy().astype(np.float64) - ref
+            assert np.abs(err).max() <= 2e-2 * np.abs(ref).max()
+            assert np.sqrt((err ** 2).mean()) <= 6e-3 * np.sqrt((ref ** 2).mean())
