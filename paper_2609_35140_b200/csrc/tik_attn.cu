@@ -181,19 +181,22 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     int my_phys = p.num_pages;                              // paged regimes: one block-table entry per lane
     auto produce_tile = [&](int it) {                       // whole warp (paged) or lane 0 (train)
         const int j = tile_first + it;
-        const int nst = kv ? KV_STAGES : KS;
-        const int st = it % nst;
-        const uint32_t use = it / nst;
+        // (no division by a run-time stage count: this code sits between a stage's release and its
+        // next request, and the issuing threads below are the pace-makers of the tensor pipe)
+        const bool two = !kv && KS == 2;
+        const int st = two ? (it & 1) : (it % KV_STAGES);
+        const uint32_t use = two ? (it >> 1) : (it / KV_STAGES);
         const uint32_t dst = (kv ? sV : sK) + st * L::TILE;
         const uint32_t full = (kv ? bar_vfull : bar_kfull) + 8 * st;
         if (MODE != MODE_TRAIN) {
             // Paged K/V: the warp reads 32 block-table entries at a time (one per lane, coalesced),
             // so the table's latency is paid once per 32 pages instead of before every tile.
-            const int tiles_per_batch = 32 / p.pages_per_tile;
-            if (it % tiles_per_batch == 0) {
-                const int lp = (128 * j) / p.page_size + lane;
+            // (page sizes are powers of two: shifts, not divisions)
+            const int tpb_mask = (32 >> p.ppt_shift) - 1;             // tiles per batch - 1
+            if ((it & tpb_mask) == 0) {
+                const int lp = ((128 * j) >> p.page_shift) + lane;
                 int ph = p.num_pages;       // out of range: the box is filled with zeros
-                if (lp * p.page_size < ctx) {
+                if ((lp << p.page_shift) < ctx) {
                     ph = (lp < p.max_blocks) ? p.block_table[static_cast<long long>(seq) * p.max_blocks + lp] : -1;
                     if (ph < 0 || ph >= p.num_pages) {
                         if (kv == 0) atomicOr(p.dev_status, TIK_DEV_BAD_BLOCK);
@@ -202,6 +205,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
                 my_phys = ph;
             }
+        }
+        // paged: lane i < pages_per_tile takes the tile's i-th page (everything that does not need
+        // the stage to be free happens before the wait; after it only the copies are issued)
+        int my_page = 0;
+        if (MODE != MODE_TRAIN) {
+            const int in_batch = it & ((32 >> p.ppt_shift) - 1);
+            my_page = __shfl_sync(0xffffffffu, my_phys, (in_batch << p.ppt_shift) + (lane & (p.pages_per_tile - 1)));
         }
         // Each stage has its own release barrier with this warp as its only waiter: a barrier
         // shared with waiters of a different lag could run two phases ahead of the slowest one,
@@ -215,15 +225,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 for (int a = 0; a < NATOM; ++a) tma_load_3d(dst + a * L::ATOM, tm, full, a * 64, kvh, row);
             }
         } else {
-            const int ppt = p.pages_per_tile;
-            const int in_batch = it % (32 / ppt);
-            for (int i = 0; i < ppt; ++i) {
-                const int phys = __shfl_sync(0xffffffffu, my_phys, in_batch * ppt + i);
-                if (lane == 0) {
-                    const uint32_t off = static_cast<uint32_t>(i * p.page_size) * 128u;
-                    for (int a = 0; a < NATOM; ++a)
-                        tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, phys);
-                }
+            __syncwarp();                                 // the expected byte count is registered first
+            if (lane < p.pages_per_tile) {
+                const uint32_t off = static_cast<uint32_t>(lane << p.page_shift) * 128u;
+                for (int a = 0; a < NATOM; ++a)
+                    tma_load_4d(dst + a * L::ATOM + off, tm, full, a * 64, 0, kvh, my_page);
             }
         }
     };
@@ -358,8 +364,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const int bz = static_cast<int>(nxt / (static_cast<long long>(gridDim.x) * gridDim.y));
                 const int ctx2 = p.ctx_lens[bz];
                 const int pos2 = bx * p.cpc * CHUNK;                 // first key position of that CTA
-                const int lp = pos2 / p.page_size + lane;
-                if (lane < KV_STAGES * p.pages_per_tile && lp < p.max_blocks && lp * p.page_size < ctx2) {
+                const int lp = (pos2 >> p.page_shift) + lane;
+                if (lane < KV_STAGES * p.pages_per_tile && lp < p.max_blocks && (lp << p.page_shift) < ctx2) {
                     const int ph = p.block_table[static_cast<long long>(bz) * p.max_blocks + lp];
                     if (ph >= 0 && ph < p.num_pages)
                         for (int a = 0; a < NATOM; ++a) tma_prefetch_l2_4d(tm, a * 64, 0, by, ph);
@@ -378,10 +384,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             const uint64_t dq1 = smem_desc_sw128(sQ + L::TILE, 0, 1024);
             for (int g = 0; g < n_steps; ++g) {
                 const int kt = pair ? (g >> 1) : g;                 // K tile of this step
-                const int st = kt % KS, b = g & 1;
+                const int st = (KS == 2) ? (kt & 1) : (kt % KV_STAGES), b = g & 1;
+                const int kuse = (KS == 2) ? (kt >> 1) : (kt / KV_STAGES);
                 // the single score buffer is free once the softmax of step g-1 holds it in registers
                 if (g >= 1) mbar_wait(bar_sempty + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_word, p.dev_status);
-                mbar_wait(bar_kfull + 8 * st, (kt / KS) & 1, abort_word, p.dev_status);
+                mbar_wait(bar_kfull + 8 * st, kuse & 1, abort_word, p.dev_status);
                 tc_fence_after();
                 const uint64_t dq = (pair && b) ? dq1 : dq0;
                 const uint64_t dk = smem_desc_sw128(sK + st * L::TILE, 0, 1024);

@@ -36,6 +36,7 @@ struct AttnParams {
     float c;                     // softmax_scale * log2(e)
     float* part_o;               // decode: [B][Hq][nchunk_max][d]
     float* part_ml;              // decode: [B][Hq][nchunk_max][4] = m, l_lo, l_hi, unused
+    int page_shift, ppt_shift;   // log2(page_size), log2(pages_per_tile)
     int nchunk_max;
     int cpc;                     // decode: consecutive chunks streamed by one CTA
     int* dev_status;

@@ -125,6 +125,8 @@ extern "C" tik_status tik_attn_decode_static(const void* q, void* o, float* lse,
     p.G = G;
     p.page_size = page_size;
     p.pages_per_tile = 128 / page_size;
+    p.page_shift = page_size == 16 ? 4 : page_size == 32 ? 5 : page_size == 64 ? 6 : 7;
+    p.ppt_shift = 7 - p.page_shift;
     p.num_pages = num_pages;
     p.c = softmax_scale * LOG2E_F;
     p.nchunk_max = nchunk;
