@@ -48,6 +48,36 @@ struct AttnSmem {
     static constexpr uint32_t ALLOC = BYTES;                      // base must be 1 KiB aligned
 };
 
+// Rarely taken paths of the softmax loops, kept out of line so that the loop bodies stay small
+// (the loops of two warpgroups, the issuing threads and the producers share one instruction cache).
+template <int D>
+__device__ __noinline__ void rescale_o_tmem(uint32_t to, float alpha) {
+#pragma unroll 1
+    for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(to + 32 * cc, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
+        tmem_st32(to + 32 * cc, v);
+    }
+}
+template <int D>
+__device__ __noinline__ void fold_o_tmem(uint32_t t_a, uint32_t t_b, FoldCoef f) {
+#pragma unroll 1
+    for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t a[32], b[32];
+        tmem_ld32(t_a + 32 * cc, a);
+        tmem_ld32(t_b + 32 * cc, b);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            a[i] = __float_as_uint(fold_value(__uint_as_float(a[i]), __uint_as_float(b[i]), f));
+        tmem_st32(t_a + 32 * cc, a);
+    }
+    tmem_wait_st();
+}
+
 template <int D, int MODE>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -468,20 +498,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 Lg_lo = fold_value(Lg_lo, l_c_lo, f);
                 Lg_hi = fold_value(Lg_hi, l_c_hi, f);
                 M_g = f.M_new;
-                if (with_o) {
-#pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
-                        uint32_t a[32], b[32];
-                        tmem_ld32(tlane + COL_OA + 32 * cc, a);
-                        tmem_ld32(tlane + COL_OB + 32 * cc, b);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            a[i] = __float_as_uint(fold_value(__uint_as_float(a[i]), __uint_as_float(b[i]), f));
-                        tmem_st32(tlane + COL_OA + 32 * cc, a);
-                    }
-                    tmem_wait_st();
-                }
+                if (with_o) fold_o_tmem<D>(tlane + COL_OA, tlane + COL_OB, f);
             }
         };
         // decode: the partial of a finished chunk; the accumulator columns [col0, col0 + ncol)
@@ -621,17 +638,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         write_partial_o(chunk_of(it - 1), 0, D);
                     } else if (!chunk_start && !__all_sync(0xffffffffu, alpha == 1.0f)) {
                         wait_pv(it - 1);
-                        const uint32_t to = tlane + col_o_of(it);
-#pragma unroll
-                        for (int cc = 0; cc < D / 32; ++cc) {
-                            uint32_t v[32];
-                            tmem_ld32(to + 32 * cc, v);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
-                            tmem_st32(to + 32 * cc, v);
-                        }
+                        rescale_o_tmem<D>(tlane + col_o_of(it), alpha);
                     }
                     tmem_wait_st();
                 }
@@ -707,16 +714,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 l_hi = __fmaf_rn(l_hi, alpha, rs_hi.total());
                 if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.0f)) {
                     // rescale this tile's accumulator (its last PV, step g-2, is complete)
-#pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
-                        uint32_t v[32];
-                        tmem_ld32(to + 32 * cc, v);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
-                        tmem_st32(to + 32 * cc, v);
-                    }
+                    rescale_o_tmem<D>(to, alpha);
                 }
                 tmem_wait_st();
                 tc_fence_before();
@@ -858,17 +856,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 } else if (!chunk_start && !__all_sync(0xffffffffu, alpha == 1.0f)) {
                     // rescale the chunk accumulator of this row
                     wait_pv(it - 1);
-                    const uint32_t to = tlane + col_o_of(it);
-#pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
-                        uint32_t v[32];
-                        tmem_ld32(to + 32 * cc, v);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            v[i] = __float_as_uint(rescale_o(__uint_as_float(v[i]), alpha));
-                        tmem_st32(to + 32 * cc, v);
-                    }
+                    rescale_o_tmem<D>(tlane + col_o_of(it), alpha);
                 }
                 tmem_wait_st();
                 // this thread closed a chunk that is not the row's last: fold its scalars here too
