@@ -147,6 +147,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tile_first = 0;
         tile_last = T0;
     } else {
+        pdl_launch_dependents();       // the combine kernel may be scheduled behind this grid's last wave
         seq = blockIdx.z;
         kvh = blockIdx.y;
         head = kvh * p.G;
@@ -954,6 +955,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 // partials (m, l_lo, l_hi, O) in ascending chunk order and normalises.
 template <int D>
 __global__ void __launch_bounds__(D) combine_kernel(const AttnParams p) {
+    pdl_wait();                        // the decode kernel's partials are complete and visible
     const int b = blockIdx.x / p.Hq;
     const int ctx = p.ctx_lens[b];
     if (ctx <= 0) return;
@@ -1042,9 +1044,18 @@ cudaError_t launch_attn(int d, int mode, dim3 grid, const CUtensorMap& tmQ, cons
 }
 
 cudaError_t launch_combine(int d, const AttnParams& p, int B, cudaStream_t stream) {
-    if (d == 128) combine_kernel<128><<<B * p.Hq, 128, 0, stream>>>(p);
-    else combine_kernel<64><<<B * p.Hq, 64, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(B) * p.Hq);
+    cfg.blockDim = dim3(d);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (d == 128) return cudaLaunchKernelEx(&cfg, combine_kernel<128>, p);
+    return cudaLaunchKernelEx(&cfg, combine_kernel<64>, p);
 }
 
 cudaError_t launch_kv_write(const void* k_new, const void* v_new, const int32_t* cu_new,

@@ -37,6 +37,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr uint32_t TMEM_COLS = 512;      // two 256-column accumulators
     constexpr uint32_t IDESC = mma_idesc_bf16(128, NB, false);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_launch_dependents();           // the finish kernel may be scheduled behind this grid's last wave
 
     // raster: bands of BAND token tiles; within a band the token tile varies fastest so the
     // CTAs in flight share one lm_head super-chunk and the band's hidden rows stay in L2
@@ -214,6 +215,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 // One thread per token: fold the super-chunk pairs in ascending order, write the result.
 __global__ void __launch_bounds__(256) logprob_finish_kernel(const LogprobParams p) {
+    pdl_wait();                        // the super-chunk pairs and target logits are complete and visible
     const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (t >= p.T) return;
     const float* ml = p.part_ml + 2 * t * p.nsuper;
@@ -250,8 +252,16 @@ cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const
     logprob_kernel<<<static_cast<unsigned>(grid), lp::THREADS, lp::ALLOC, stream>>>(tmA, tmB, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    logprob_finish_kernel<<<static_cast<unsigned>((p.T + 255) / 256), 256, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>((p.T + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, logprob_finish_kernel, p);
 }
 
 }  // namespace tik

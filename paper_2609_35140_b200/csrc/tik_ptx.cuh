@@ -75,6 +75,15 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity,
     }
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may start while its
+// predecessor in the stream still runs: its CTAs are scheduled once every CTA of the predecessor
+// has executed launch_dependents (or exited), and pdl_wait() blocks until the predecessor has
+// completed and its writes are visible.  Used for the small second kernel of a two-kernel call
+// (split-KV combine, log-prob finish) so that its launch latency hides under the first one's tail.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
