@@ -91,10 +91,11 @@ struct LogprobParams {
     float* z_target;             // [T]
     int64_t T;
     int H, V, nsuper;
+    int spc;                     // consecutive 1024-column super-chunks walked by one CTA
     float inv_temperature;
     int* dev_status;
 };
-cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p,
+cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p, bool pair,
                            cudaStream_t stream);
 
 struct NormParams {
@@ -113,11 +114,11 @@ struct LinearParams {
     __nv_bfloat16* y;            // [T][N]
     int64_t T;
     int K, N, nsuper;
-    int super_cols;              // output columns per CTA: 256, 512 or 1024
+    int super_cols;              // output columns per CTA: 256 .. 4096 (a power of two)
     int* dev_status;
 };
-cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const LinearParams& p,
-                          cudaStream_t stream);
+cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                          const LinearParams& p, cudaStream_t stream);
 
 struct BwdParams {
     const int32_t* cu_seqlens;   // [S+1]

@@ -1,10 +1,10 @@
 // Dense linear layer y = x W^T (bf16 in, fp32 accumulation in TMEM, bf16 out) for sm_100a: the
 // FFN projections of the unified operator set.  Same machinery as the log-probability GEMM: one
-// CTA = (128-row tile, super-chunk of 256 to 1024 output columns); a TMA warp streams 64-wide K slices of x and W
+// CTA = (128-row tile, super-chunk of 256 to 4096 output columns); a TMA warp streams 64-wide K slices of x and W
 // through a four-stage shared-memory ring, an MMA warp accumulates the whole K range in ascending
 // order into one of two 256-column TMEM accumulators (M128 x N256 x K16, no split-K), and four
-// epilogue warps (one thread per row) round the accumulator to bf16 and store it while the next
-// 256 columns are being accumulated.  An output element is one fixed chain of MMAs over K, so it
+// epilogue warps (one thread per row) round the accumulator to bf16 and send it out through
+// shared memory and tiled TMA stores while the next 256 columns are being accumulated.  An output element is one fixed chain of MMAs over K, so it
 // depends on its x row and its W row only: a row gives the same bits whether it is computed alone
 // (decode) or inside a long batch (prefill, policy update).
 #include "tik_core.cuh"
@@ -16,11 +16,12 @@ namespace tik {
 namespace lin {
 constexpr int STAGES = 4;
 constexpr int NB = 256;                      // output columns per MMA
-constexpr int SUPER_MAX = 1024;              // output columns per CTA (256, 512 or 1024, chosen per launch)
 constexpr uint32_t A_BYTES = 128 * 128;      // 128 rows x 64 bf16
 constexpr uint32_t B_BYTES = NB * 128;       // 256 W rows x 64 bf16
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr uint32_t OFF_BAR = STAGES * STAGE_BYTES;
+constexpr uint32_t STG_BYTES = 128 * 128;    // output staging: 128 rows x 64 bf16, two buffers
+constexpr uint32_t OFF_STG = STAGES * STAGE_BYTES;
+constexpr uint32_t OFF_BAR = OFF_STG + 2 * STG_BYTES;
 constexpr uint32_t BYTES = OFF_BAR + 256;
 constexpr uint32_t ALLOC = BYTES + 1024;
 constexpr int BAND = 32;                     // row tiles per L2 band
@@ -29,7 +30,7 @@ constexpr int THREADS = 192;                 // warp 0 TMA, warp 1 MMA, warps 2.
 
 __global__ void __launch_bounds__(lin::THREADS, 1)
 linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-              const LinearParams p) {
+              const __grid_constant__ CUtensorMap tmY, const LinearParams p) {
     using namespace lin;
     constexpr uint32_t TMEM_COLS = 512;      // two 256-column accumulators
     constexpr uint32_t IDESC = mma_idesc_bf16(128, NB, false);
@@ -75,6 +76,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
+        tma_prefetch_desc(&tmY);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
@@ -127,40 +129,52 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5)
+        // Thread per row: 64 columns at a time go from TMEM to a 128B-swizzled staging tile in
+        // shared memory and leave as one tiled TMA store of 128 rows x 128 bytes (row-by-row
+        // 16-byte stores from 128 threads cost a third of the kernel on wide outputs).  The store
+        // clips at the tensor's bounds, so rows past T and columns past N need no guard.  Two
+        // staging tiles alternate; the issuing thread lets at most one store group read behind it.
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
         const int row = quarter * 32 + lane;
-        const long long t = static_cast<long long>(row0) + row;
-        const bool row_valid = t < p.T;
-        __nv_bfloat16* yrow = p.y + t * p.N;
+        uint32_t piece = 0;
         for (int nt = 0; nt < n_nt; ++nt) {
             const int buf = nt & 1;
             mbar_wait(bar_acc_full + 8 * buf, (nt >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
             const int col0 = col_base + nt * NB;
             const uint32_t taddr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * NB;
-#pragma unroll 2
-            for (int cc = 0; cc < NB / 32; ++cc) {
-                if (col0 + 32 * cc >= p.N) break;              // warp-uniform: columns past N
-                uint32_t v[32];
-                tmem_ld32(taddr + 32 * cc, v);
+#pragma unroll 1
+            for (int q = 0; q < NB / 64; ++q, ++piece) {
+                if (col0 + 64 * q >= p.N) break;               // uniform: columns past N
+                uint32_t v[64];
+                tmem_ld32(taddr + 64 * q, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                tmem_ld32(taddr + 64 * q + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
                 tmem_wait_ld();
-                if (row_valid) {
+                uint8_t* stg = smem + OFF_STG + (piece & 1) * STG_BYTES;
+                // the store that last read this staging tile (two pieces ago) has finished reading
+                if (warp == 2 && lane == 0) tma_store_wait_read1();
+                named_bar_sync(1, 128);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int col = col0 + 32 * cc + 8 * i;
-                        if (col < p.N)                         // N is a multiple of 8
-                            *reinterpret_cast<uint4*>(yrow + col) = make_uint4(
-                                pack_bf16x2(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
-                                pack_bf16x2(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
-                                pack_bf16x2(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
-                                pack_bf16x2(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
-                    }
+                for (int c16 = 0; c16 < 8; ++c16) {
+                    const uint4 val = make_uint4(
+                        pack_bf16x2(__uint_as_float(v[8 * c16]), __uint_as_float(v[8 * c16 + 1])),
+                        pack_bf16x2(__uint_as_float(v[8 * c16 + 2]), __uint_as_float(v[8 * c16 + 3])),
+                        pack_bf16x2(__uint_as_float(v[8 * c16 + 4]), __uint_as_float(v[8 * c16 + 5])),
+                        pack_bf16x2(__uint_as_float(v[8 * c16 + 6]), __uint_as_float(v[8 * c16 + 7])));
+                    *reinterpret_cast<uint4*>(stg + row * 128 + ((c16 ^ (row & 7)) << 4)) = val;
+                }
+                fence_proxy_async_smem();
+                named_bar_sync(1, 128);
+                if (warp == 2 && lane == 0) {
+                    tma_store_2d(&tmY, smem_u32(stg), col0 + 64 * q, row0);
+                    tma_store_commit();
                 }
             }
             // all TMEM reads of this accumulator are done: hand it back to the MMA warp
             tc_fence_before();
             mbar_arrive(bar_acc_empty + 8 * buf);
         }
+        if (warp == 2 && lane == 0) tma_store_wait_read();     // shared memory stays valid until the last read
     }
 
     if (*abort_word) {   // let copies and MMAs in flight finish before shared memory and TMEM are released
@@ -173,8 +187,8 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const LinearParams& p,
-                          cudaStream_t stream) {
+cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                          const LinearParams& p, cudaStream_t stream) {
     if (p.T <= 0) return cudaSuccess;
     static bool configured = false;
     if (!configured) {
@@ -186,7 +200,7 @@ cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const 
     const long long ntile = (p.T + 127) / 128;
     const long long nband = (ntile + lin::BAND - 1) / lin::BAND;
     const long long grid = nband * lin::BAND * p.nsuper;
-    linear_kernel<<<static_cast<unsigned>(grid), lin::THREADS, lin::ALLOC, stream>>>(tmA, tmB, p);
+    linear_kernel<<<static_cast<unsigned>(grid), lin::THREADS, lin::ALLOC, stream>>>(tmA, tmB, tmY, p);
     return cudaGetLastError();
 }
 

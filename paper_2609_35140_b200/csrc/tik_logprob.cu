@@ -18,41 +18,56 @@
 namespace tik {
 
 namespace lp {
-constexpr int STAGES = 4;
 constexpr int NB = 256;                      // vocabulary columns per MMA (two log-sum-exp tiles)
 constexpr uint32_t A_BYTES = 128 * 128;      // 128 token rows x 64 bf16
-constexpr uint32_t B_BYTES = NB * 128;       // 256 vocab rows x 64 bf16
-constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr uint32_t OFF_BAR = STAGES * STAGE_BYTES;
-constexpr uint32_t BYTES = OFF_BAR + 256;
-constexpr uint32_t ALLOC = BYTES + 1024;
-constexpr int BAND = 32;                     // token tiles per L2 band
+constexpr int BAND = 32;                     // token tiles per L2 band (even: CTA pairs stay inside a band)
 constexpr int THREADS = 192;                 // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+// PAIR: two CTAs on neighbouring SMs (a cluster of two) share every MMA: M = 256 token rows, each
+// CTA stages its own 128 token rows and half (128 rows) of the 256 lm_head rows, so a stage is
+// 32 KiB instead of 48 and the B operand crosses shared memory once per 256 token rows.
+template <bool PAIR>
+struct Cfg {
+    static constexpr int STAGES = PAIR ? 6 : 4;
+    static constexpr uint32_t B_BYTES = (PAIR ? NB / 2 : NB) * 128;
+    static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr uint32_t OFF_BAR = STAGES * STAGE_BYTES;
+    static constexpr uint32_t BYTES = OFF_BAR + 256;
+    static constexpr uint32_t ALLOC = BYTES + 1024;
+};
 }  // namespace lp
 
+template <bool PAIR>
 __global__ void __launch_bounds__(lp::THREADS, 1)
 logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const LogprobParams p) {
     using namespace lp;
+    using C = Cfg<PAIR>;
+    constexpr int STAGES = C::STAGES;
+    constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES, OFF_BAR = C::OFF_BAR;
     constexpr uint32_t TMEM_COLS = 512;      // two 256-column accumulators
-    constexpr uint32_t IDESC = mma_idesc_bf16(128, NB, false);
+    constexpr uint32_t IDESC = mma_idesc_bf16(PAIR ? 256 : 128, NB, false);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;     // 0 = the CTA that issues the pair's MMAs
     pdl_launch_dependents();           // the finish kernel may be scheduled behind this grid's last wave
 
     // raster: bands of BAND token tiles; within a band the token tile varies fastest so the
     // CTAs in flight share one lm_head super-chunk and the band's hidden rows stay in L2
     const int ntile = static_cast<int>((p.T + 127) / 128);
-    const long long per_band = static_cast<long long>(BAND) * p.nsuper;
+    const int ngroup = (p.nsuper + p.spc - 1) / p.spc;      // a CTA walks spc consecutive super-chunks
+    const long long per_band = static_cast<long long>(BAND) * ngroup;
     const int band = static_cast<int>(blockIdx.x / per_band);
     const int band_tiles = min(BAND, ntile - band * BAND);
     const long long rem = blockIdx.x - band * per_band;
     // (blockIdx.x enumerates BAND * nsuper slots per band; slots beyond a short last band exit)
-    const int sup = static_cast<int>(rem / BAND);
+    const int sup0 = static_cast<int>(rem / BAND) * p.spc;
+    const int n_sp = min(p.spc, p.nsuper - sup0);
     const int tile_in_band = static_cast<int>(rem % BAND);
-    if (tile_in_band >= band_tiles) return;
+    // (a pair leaves only together: a lone tile at the end of T keeps its partner, whose rows lie
+    // past T, arrive as zeros and are never stored)
+    if ((PAIR ? (tile_in_band & ~1) : tile_in_band) >= band_tiles) return;
     const int tok0 = (band * BAND + tile_in_band) * 128;
-    const int col_base = sup * LP_SUPER;
-    const int n_nt = min(LP_SUPER / NB, (p.V - col_base + NB - 1) / NB);   // 256-column steps
+    // 256-column accumulator steps of super-chunk sup0 + sp
+    auto n_nt_of = [&](int sp) { return min(LP_SUPER / NB, (p.V - (sup0 + sp) * LP_SUPER + NB - 1) / NB); };
     const int n_kb = p.H / 64;
 
     extern __shared__ uint8_t smem_raw[];
@@ -74,7 +89,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
-            mbar_init(bar_acc_empty + 8 * b, 128);
+            mbar_init(bar_acc_empty + 8 * b, PAIR ? 256 : 128);   // the epilogue threads of every CTA of the pair
         }
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
         fence_barrier_init();
@@ -82,38 +97,60 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tma_prefetch_desc(&tmB);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
-        tmem_relinquish();
+        if (PAIR) {
+            tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();            // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // the leader's copies of the barriers that both CTAs signal (shared::cluster addresses)
+    const uint32_t lead_full = PAIR ? mapa_cluster(bar_full, 0) : bar_full;
+    const uint32_t lead_acc_empty = PAIR ? mapa_cluster(bar_acc_empty, 0) : bar_acc_empty;
+    const uint32_t peer_empty = PAIR ? mapa_cluster(bar_empty, 1) : bar_empty;
+    const uint32_t peer_acc_full = PAIR ? mapa_cluster(bar_acc_full, 1) : bar_acc_full;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int nt = 0; nt < n_nt; ++nt) {
-                const int col0 = col_base + nt * NB;
+            for (int sp = 0; sp < n_sp; ++sp)
+            for (int nt = 0; nt < n_nt_of(sp); ++nt) {
+                const int col0 = (sup0 + sp) * LP_SUPER + nt * NB;
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
                     const int s = it % STAGES;
                     const uint32_t use = it / STAGES;
                     if (use > 0) mbar_wait(bar_empty + 8 * s, (use - 1) & 1, abort_word, p.dev_status);
-                    mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
-                    tma_load_2d(sbase + s * STAGE_BYTES, &tmA, bar_full + 8 * s, kb * 64, tok0);
-                    tma_load_2d(sbase + s * STAGE_BYTES + A_BYTES, &tmB, bar_full + 8 * s, kb * 64, col0);
+                    if (PAIR) {
+                        // both CTAs' bytes are counted on the leader's barrier, which the leader arms;
+                        // a peer copy that lands first only makes the count negative for a moment
+                        if (rank == 0) mbar_expect_tx(bar_full + 8 * s, 2 * STAGE_BYTES);
+                        tma_load_2d_pair(sbase + s * STAGE_BYTES, &tmA, lead_full + 8 * s, kb * 64, tok0);
+                        tma_load_2d_pair(sbase + s * STAGE_BYTES + A_BYTES, &tmB, lead_full + 8 * s, kb * 64,
+                                         col0 + 128 * static_cast<int>(rank));
+                    } else {
+                        mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
+                        tma_load_2d(sbase + s * STAGE_BYTES, &tmA, bar_full + 8 * s, kb * 64, tok0);
+                        tma_load_2d(sbase + s * STAGE_BYTES + A_BYTES, &tmB, bar_full + 8 * s, kb * 64, col0);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            uint32_t it = 0;
-            for (int nt = 0; nt < n_nt; ++nt) {
-                const int buf = nt & 1;
-                const uint32_t use = nt >> 1;
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, acc = 0;              // acc counts accumulator steps across super-chunks
+            for (int sp = 0; sp < n_sp; ++sp)
+            for (int nt = 0; nt < n_nt_of(sp); ++nt, ++acc) {
+                const int buf = acc & 1;
+                const uint32_t use = acc >> 1;
                 if (use > 0) mbar_wait(bar_acc_empty + 8 * buf, (use - 1) & 1, abort_word, p.dev_status);
                 tc_fence_after();
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
@@ -122,11 +159,23 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     mbar_wait(bar_full + 8 * s, (it / STAGES) & 1, abort_word, p.dev_status);
                     tc_fence_after();
                     const uint32_t a0 = sbase + s * STAGE_BYTES, b0 = a0 + A_BYTES;
-                    mma_ss_chain4(tmem + buf * NB, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
-                                  IDESC, kb ? 1u : 0u);
-                    mma_commit(bar_empty + 8 * s);
+                    if (PAIR) {
+                        mma_ss_chain4_pair(tmem + buf * NB, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
+                                           IDESC, kb ? 1u : 0u);
+                        mma_commit_pair(bar_empty + 8 * s);          // the stage is free in this CTA ...
+                        mma_commit_pair(peer_empty + 8 * s);         // ... and in the peer
+                    } else {
+                        mma_ss_chain4(tmem + buf * NB, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
+                                      IDESC, kb ? 1u : 0u);
+                        mma_commit(bar_empty + 8 * s);
+                    }
                 }
-                mma_commit(bar_acc_full + 8 * buf);
+                if (PAIR) {
+                    mma_commit_pair(bar_acc_full + 8 * buf);
+                    mma_commit_pair(peer_acc_full + 8 * buf);
+                } else {
+                    mma_commit(bar_acc_full + 8 * buf);
+                }
             }
         }
     } else {
@@ -137,11 +186,14 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool row_valid = t < p.T;
         const int target = row_valid ? p.target[t] : -1;
         const float it_scale = p.inv_temperature;
+        uint32_t acc = 0;
+        for (int sp = 0; sp < n_sp; ++sp) {
+        const int col_base = (sup0 + sp) * LP_SUPER;
         float M = -CUDART_INF_F, Lsum = 0.0f;
         bool first = true;
-        for (int nt = 0; nt < n_nt; ++nt) {
-            const int buf = nt & 1;
-            mbar_wait(bar_acc_full + 8 * buf, (nt >> 1) & 1, abort_word, p.dev_status);
+        for (int nt = 0; nt < n_nt_of(sp); ++nt, ++acc) {
+            const int buf = acc & 1;
+            mbar_wait(bar_acc_full + 8 * buf, (acc >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
 #pragma unroll 1
             for (int half = 0; half < NB / LP_TILE; ++half) {
@@ -195,11 +247,13 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             // all TMEM reads of this accumulator are done: hand it back to the MMA warp
             tc_fence_before();
-            mbar_arrive(bar_acc_empty + 8 * buf);
+            if (PAIR) mbar_arrive_cluster(lead_acc_empty + 8 * buf);
+            else mbar_arrive(bar_acc_empty + 8 * buf);
         }
         if (row_valid) {
-            p.part_ml[2 * (t * p.nsuper + sup)] = M;
-            p.part_ml[2 * (t * p.nsuper + sup) + 1] = Lsum;
+            p.part_ml[2 * (t * p.nsuper + sup0 + sp)] = M;
+            p.part_ml[2 * (t * p.nsuper + sup0 + sp) + 1] = Lsum;
+        }
         }
     }
 
@@ -210,7 +264,11 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
+    if (PAIR) cluster_sync_all();            // neither CTA leaves while the other may still touch it
+    if (warp == 1) {
+        if (PAIR) tmem_dealloc_pair(tmem, TMEM_COLS);
+        else tmem_dealloc(tmem, TMEM_COLS);
+    }
 }
 
 // One thread per token: fold the super-chunk pairs in ascending order, write the result.
@@ -236,21 +294,41 @@ __global__ void __launch_bounds__(256) logprob_finish_kernel(const LogprobParams
     }
 }
 
-cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p,
-                           cudaStream_t stream) {
-    if (p.T <= 0) return cudaSuccess;
+template <bool PAIR>
+static cudaError_t launch_logprob_main(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p,
+                                       cudaStream_t stream) {
+    using C = lp::Cfg<PAIR>;
+    auto kern = logprob_kernel<PAIR>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(logprob_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(lp::ALLOC));
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(C::ALLOC));
         if (e != cudaSuccess) return e;
         configured = true;
     }
     const long long ntile = (p.T + 127) / 128;
     const long long nband = (ntile + lp::BAND - 1) / lp::BAND;
-    const long long grid = nband * lp::BAND * p.nsuper;
-    logprob_kernel<<<static_cast<unsigned>(grid), lp::THREADS, lp::ALLOC, stream>>>(tmA, tmB, p);
-    cudaError_t e = cudaGetLastError();
+    const long long grid = nband * lp::BAND * ((p.nsuper + p.spc - 1) / p.spc);   // even: BAND is
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(lp::THREADS);
+    cfg.dynamicSmemBytes = C::ALLOC;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
+}
+
+// pair = true: tmB must have a box of 128 rows (each CTA of a pair stages half of the 256 columns)
+cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p, bool pair,
+                           cudaStream_t stream) {
+    if (p.T <= 0) return cudaSuccess;
+    cudaError_t e = pair ? launch_logprob_main<true>(tmA, tmB, p, stream) : launch_logprob_main<false>(tmA, tmB, p, stream);
     if (e != cudaSuccess) return e;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
