@@ -37,7 +37,7 @@ METRIC = "summed_attention_ms"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch of the dominant kernel from one ncu capture (profiles/), keyed by
 # workload index; None until captured.
-NCU_TRAFFIC_BYTES = {1: 2905034344}     # logprob_kernel on workload 1: 2.872 GB read + 30.4 MB written
+NCU_TRAFFIC_BYTES = {1: 3485940960}     # logprob_kernel on workload 1: 3.454 GB read + 32.2 MB written
 
 
 def load_peaks():
@@ -550,7 +550,7 @@ def main():
     dom_name = max(("train_fwd", "prefill", "logprob"), key=lambda n: rooflines[n]["ms"])
     dom = rooflines[dom_name]
     roofline = {"kernel": {"train_fwd": "attn_kernel<128,train>", "prefill": "attn_kernel<128,prefill>",
-                           "logprob": "logprob_kernel"}[dom_name],
+                           "logprob": "logprob_kernel<pair>"}[dom_name],
                 "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
                 "frac": dom["frac"], "traffic": NCU_TRAFFIC_BYTES.get(w.index),
                 "peak_source": "of %s (%s bf16 peak: median SM clock %s of %s MHz in the timed region)" % (
