@@ -93,6 +93,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     constexpr uint32_t IDESC_PV = mma_idesc_bf16(128, D, true);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // Launched with programmatic stream serialization: the grid may be scheduled while the kernel
+    // before it in the stream (typically the cache write or the pre-attention step of the same
+    // call sequence) is still draining; nothing of this kernel's input is read before this wait.
+    pdl_wait();
 
     // ---------------------------------------------------------------- work item
     // Train / prefill: query tiles are aligned to absolute positions.  Tiles 0..15 (their KV
@@ -987,6 +991,7 @@ kv_write_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new
                 uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
                 const int32_t* __restrict__ block_table, int max_blocks, int S, int Hkv,
                 int vec_per_head /* d*2/16 */, int page_size, int num_pages, int* dev_status) {
+    pdl_launch_dependents();       // an attention kernel launched next may be scheduled behind this grid
     const int token = blockIdx.x;
     int lo = 0, hi = S;            // find s with cu_new[s] <= token < cu_new[s+1]
     while (hi - lo > 1) {
@@ -1027,8 +1032,17 @@ static cudaError_t launch_attn_t(dim3 grid, const CUtensorMap& tmQ, const CUtens
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, ATTN_THREADS, AttnSmem<D>::ALLOC, stream>>>(tmQ, tmK, tmV, p);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(ATTN_THREADS);
+    cfg.dynamicSmemBytes = AttnSmem<D>::ALLOC;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, tmQ, tmK, tmV, p);
 }
 
 cudaError_t launch_attn(int d, int mode, dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK,

@@ -57,6 +57,7 @@ template <int D>
 __global__ void __launch_bounds__(PREP_WARPS * 32, PREP_MIN_CTAS) prep_kernel(const PrepParams p) {
     constexpr int EP = D / 32;
     constexpr int VPH = D * 2 / 16;             // 16-byte pieces of one V row
+    pdl_launch_dependents();       // an attention kernel launched next may be scheduled behind this grid
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane >> 4, l16 = lane & 15;
     const long long token = static_cast<long long>(blockIdx.x) * PREP_WARPS + warp;   // one warp per token
