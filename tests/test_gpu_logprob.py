@@ -80,6 +80,22 @@ def test_batch_shape_invariance(tik):
         assert count_diff(full[a:b], part) == 0, (a, b)
 
 
+def test_two_bands_several_super_chunks_per_cta(tik):
+    """More than one band of 32 token tiles (the second one a single, partner-less tile) and enough
+    work that a CTA walks two super-chunks: sampled rows against the oracle, slices bit for bit."""
+    T, H, V = 128 * 40 + 70, 64, 32768 + 11
+    hidden, W, target = _inputs(T, H, V, 4321, 0.5)
+    target[:4] = torch.tensor([0, V - 1, 32767, 32768], dtype=torch.int32)
+    lp = tik.tik_token_logprob(hidden, W, target)
+    rows = torch.tensor([0, 1, 2, 3, 127, 128, 4095, 4096, 5119, 5120, T - 1] + list(range(900, 5000, 97)), device="cuda")
+    ref, _ = _oracle(hidden[rows], W, target[rows])
+    assert np.abs(lp[rows].cpu().numpy() - ref).max() <= LOGPROB_TOL
+    assert bool(torch.isfinite(lp).all())
+    for a, b in [(5120, T), (4000, 4100), (T - 1, T)]:
+        part = tik.tik_token_logprob(hidden[a:b].contiguous(), W, target[a:b].contiguous())
+        assert count_diff(lp[a:b], part) == 0, (a, b)
+
+
 def test_bad_target_is_nan_and_flagged(tik):
     T, H, V = 8, 64, 100
     hidden, W, target = _inputs(T, H, V, 9)
