@@ -3,7 +3,7 @@
 // Deterministic by construction: no atomics and no split accumulation.  Two launches of one
 // kernel body recompute the score tiles and differ in which side stays resident:
 //   DQ  mode: a CTA owns one 128-row query tile of one (sequence, head) and walks the KV tiles
-//             0..i:      S = Q_i K_j^T, dP = dO_i V_j^T, dS = P o (dP - delta) * scale,
+//             0..i:      S = Q_i K_j^T, dP = dO_i V_j^T, dS = P o (dP - delta),
 //             dQ_i += dS K_j                                     (accumulator in TMEM)
 //   DKV mode: a CTA owns one 128-row KV tile of one (sequence, KV head) and walks the query
 //             tiles i >= j of the G query heads of that KV head, one after the other:
@@ -12,10 +12,11 @@
 // (a small kernel of its own).  All five products run on tcgen05: the two score products with
 // both operands in shared memory (TMA, 128B swizzle), the gradient products with the bf16
 // weights P / dS read from TMEM, written there in place of the fp32 scores they came from.
-// One TMA warp, one MMA-issuing warp, and two element-wise warpgroups (one thread per tile row
-// each).  A step's 128 streamed rows are handled as two halves of 64: warpgroup h turns the score
-// columns of half h into weights while the tensor pipe runs the gradient product of the other
-// half and the score product of the next step, so MMAs and element-wise work overlap.
+// One TMA warp, one MMA-issuing warp, and sixteen element-wise warps.  A step's 128 streamed rows
+// are handled as two halves of 64: the eight warps of half h (two threads per tile row, 32
+// columns each) turn the half's score columns into weights while the tensor pipe runs the
+// gradient product of the other half and the score product of the next step, so MMAs and
+// element-wise work overlap and the element-wise latency of a half stays short.
 // Every wait is bounded and raises TIK_DEV_WAIT_EXPIRED instead of hanging.
 #include "tik_core.cuh"
 #include "tik_internal.h"
@@ -24,7 +25,7 @@
 namespace tik {
 
 enum { BWD_DQ = 0, BWD_DKV = 1 };
-constexpr int BWD_THREADS = 320;     // warp 0 TMA, warp 1 MMA, warps 2-9 element-wise (two per tile row)
+constexpr int BWD_THREADS = 576;     // warp 0 TMA, warp 1 MMA, warps 2-17 element-wise (four threads per tile row)
 constexpr int BWD_STAGES = 2;
 
 template <int D>
@@ -100,7 +101,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_tfull + 8 * i, 1);
-            mbar_init(bar_efull + 8 * i, 4);
+            mbar_init(bar_efull + 8 * i, 8);
         }
         mbar_init(bar_acc, 1);
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
@@ -207,8 +208,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // ------------------------------------------------------------ element-wise warps
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
         const int r = quarter * 32 + lane;                 // tile row == TMEM lane
-        const int hlf = (warp - 2) >> 2;                   // which 64 columns of the row this thread owns
-        const int et = ((warp - 2) & 3) * 32 + lane;       // 0..127 within the thread's group of four warps
+        const int hlf = (warp - 2) >> 3;                   // which half (64 streamed rows) this thread works on
+        const int sub = ((warp - 2) >> 2) & 1;             // which 32 of the half's 64 columns
+        const int et = ((warp - 2) & 7) * 32 + lane;       // 0..255 within the half's eight warps
         const uint32_t tlane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const int row_abs = 128 * own + r;                 // position of this row in the sequence
         const float c = p.c;                               // scale * log2(e)
@@ -241,7 +243,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 my_sc[2 * et] = l2;
                 my_sc[2 * et + 1] = dl;
             }
-            named_bar_sync(1 + hlf, 128);
+            named_bar_sync(1 + hlf, 256);
         }
         for (int t = 0; t < n_steps; ++t) {
             float nl2 = 0.0f, ndl = 0.0f;
@@ -251,44 +253,66 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tc_fence_after();
             // column cc of the half is masked for this row when it lies in the row's future (DQ: key
             // after query; DKV: query before key) or, DKV, past the end of the sequence
-            const int col0_abs = 128 * step_tile(t) + 64 * hlf;
+            const int col0_abs = 128 * step_tile(t) + 64 * hlf + 32 * sub;
             {
-                uint32_t s_[64], d_[64];
-                tmem_ld32(tlane + COL_T1 + 64 * hlf, *reinterpret_cast<uint32_t(*)[32]>(&s_[0]));
-                tmem_ld32(tlane + COL_T1 + 64 * hlf + 32, *reinterpret_cast<uint32_t(*)[32]>(&s_[32]));
-                tmem_ld32(tlane + COL_T2 + 64 * hlf, *reinterpret_cast<uint32_t(*)[32]>(&d_[0]));
-                tmem_ld32(tlane + COL_T2 + 64 * hlf + 32, *reinterpret_cast<uint32_t(*)[32]>(&d_[32]));
+                uint32_t s_[32], d_[32];
+                tmem_ld32(tlane + COL_T1 + 64 * hlf + 32 * sub, s_);
+                tmem_ld32(tlane + COL_T2 + 64 * hlf + 32 * sub, d_);
                 tmem_wait_ld();
-                uint32_t pk[32], dk_[32];
+                // the weights go in place of the half's scores: its first 32 columns, which the
+                // threads of sub-block 0 are reading until they have passed this barrier
+                named_bar_sync(3 + hlf, 256);
+                uint32_t pk[16], dk_[16];
+                // only the diagonal tile and (DKV) the sequence's last query tile have masked columns;
+                // everywhere else the two-wide path runs without compares and selects
+                const bool any_mask = (step_tile(t) == own) || (MODE == BWD_DKV && col0_abs + 32 > len);
+                if (!any_mask) {
 #pragma unroll
-                for (int i = 0; i < 64; i += 2) {
-                    float pv[2], dsv[2];
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int cc = i + e;
-                        const int col_abs = col0_abs + cc;
-                        bool masked;
-                        float l2, dl;
+                    for (int i = 0; i < 32; i += 2) {
+                        float nl2_0, nl2_1, ndl0, ndl1;
                         if (MODE == BWD_DQ) {
-                            masked = col_abs > row_abs;
-                            l2 = row_l2;
-                            dl = row_dl;
+                            nl2_0 = nl2_1 = -row_l2;
+                            ndl0 = ndl1 = -row_dl;
                         } else {
-                            masked = (row_abs > col_abs) || (col_abs >= len);
-                            const float2 sc2 = csc[cc];
-                            l2 = sc2.x;
-                            dl = sc2.y;
+                            const float4 sc4 = *reinterpret_cast<const float4*>(&csc[32 * sub + i]);   // (l2, dl) x 2
+                            nl2_0 = -sc4.x, ndl0 = -sc4.y, nl2_1 = -sc4.z, ndl1 = -sc4.w;
                         }
-                        const float pe = bwd_p(__uint_as_float(s_[i + e]), c, l2);
-                        pv[e] = masked ? 0.0f : pe;
-                        dsv[e] = masked ? 0.0f : bwd_ds(pe, __uint_as_float(d_[i + e]), dl, p.scale);
+                        float p0, p1, ds0, ds1;
+                        bwd_pds_x2(__uint_as_float(s_[i]), __uint_as_float(s_[i + 1]), __uint_as_float(d_[i]),
+                                   __uint_as_float(d_[i + 1]), c, nl2_0, nl2_1, ndl0, ndl1, p0, p1, ds0, ds1);
+                        pk[i >> 1] = pack_bf16x2(p0, p1);
+                        dk_[i >> 1] = pack_bf16x2(ds0, ds1);
                     }
-                    pk[i >> 1] = pack_bf16x2(pv[0], pv[1]);
-                    dk_[i >> 1] = pack_bf16x2(dsv[0], dsv[1]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float pv[2], dsv[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int cc = i + e;
+                            const int col_abs = col0_abs + cc;
+                            bool masked;
+                            float l2, dl;
+                            if (MODE == BWD_DQ) {
+                                masked = col_abs > row_abs;
+                                l2 = row_l2;
+                                dl = row_dl;
+                            } else {
+                                masked = (row_abs > col_abs) || (col_abs >= len);
+                                const float2 sc2 = csc[32 * sub + cc];
+                                l2 = sc2.x;
+                                dl = sc2.y;
+                            }
+                            const float pe = bwd_p(__uint_as_float(s_[i + e]), c, l2);
+                            pv[e] = masked ? 0.0f : pe;
+                            dsv[e] = masked ? 0.0f : bwd_ds(pe, __uint_as_float(d_[i + e]), dl);
+                        }
+                        pk[i >> 1] = pack_bf16x2(pv[0], pv[1]);
+                        dk_[i >> 1] = pack_bf16x2(dsv[0], dsv[1]);
+                    }
                 }
-                // the weights go in place of the half's own scores (its first 32 columns)
-                if (MODE == BWD_DKV) tmem_st32(tlane + COL_T1 + 64 * hlf, pk);
-                tmem_st32(tlane + COL_T2 + 64 * hlf, dk_);
+                if (MODE == BWD_DKV) tmem_st16(tlane + COL_T1 + 64 * hlf + 16 * sub, pk);
+                tmem_st16(tlane + COL_T2 + 64 * hlf + 16 * sub, dk_);
             }
             tmem_wait_st();
             if (MODE == BWD_DKV) {
@@ -298,7 +322,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     my_sc[((t + 1) & 1) * 128 + 2 * et] = nl2;
                     my_sc[((t + 1) & 1) * 128 + 2 * et + 1] = ndl;
                 }
-                named_bar_sync(1 + hlf, 128);
+                named_bar_sync(1 + hlf, 256);
             }
             tc_fence_before();
             __syncwarp();
@@ -307,7 +331,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // ---- epilogue: fp32 accumulators -> bf16 rows
         mbar_wait(bar_acc, 0, abort_word, p.dev_status);
         tc_fence_after();
-        const bool valid = row_abs < len;
+        const bool valid = row_abs < len && sub == 0;     // one thread per (row, column half) stores
         const long long tok = static_cast<long long>(tok0) + row_abs;
         __nv_bfloat16* out1 = (MODE == BWD_DQ) ? p.dq + (tok * p.Hq + head) * D : p.dk + (tok * p.Hkv + kvh) * D;
         __nv_bfloat16* out2 = p.dv + (tok * p.Hkv + kvh) * D;
@@ -315,6 +339,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int which = 0; which < (MODE == BWD_DKV ? 2 : 1); ++which) {
             const uint32_t col = which ? COL_A2 : COL_A1;
             __nv_bfloat16* out = which ? out2 : out1;
+            const float osc = which ? 1.0f : p.scale;          // dQ, dK carry the softmax scale; dV does not
 #pragma unroll
             for (int cc = hlf * (D / 64); cc < (hlf + 1) * (D / 64); ++cc) {
                 uint32_t v[32];
@@ -324,10 +349,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
                         reinterpret_cast<uint4*>(out + 32 * cc)[i] = make_uint4(
-                            pack_bf16x2(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
-                            pack_bf16x2(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
-                            pack_bf16x2(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
-                            pack_bf16x2(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
+                            pack_bf16x2(__fmul_rn(__uint_as_float(v[8 * i]), osc), __fmul_rn(__uint_as_float(v[8 * i + 1]), osc)),
+                            pack_bf16x2(__fmul_rn(__uint_as_float(v[8 * i + 2]), osc), __fmul_rn(__uint_as_float(v[8 * i + 3]), osc)),
+                            pack_bf16x2(__fmul_rn(__uint_as_float(v[8 * i + 4]), osc), __fmul_rn(__uint_as_float(v[8 * i + 5]), osc)),
+                            pack_bf16x2(__fmul_rn(__uint_as_float(v[8 * i + 6]), osc), __fmul_rn(__uint_as_float(v[8 * i + 7]), osc)));
                 }
             }
         }

@@ -242,10 +242,31 @@ __device__ __forceinline__ float swiglu_value(float g, float u) {
 }
 
 // ---- attention backward: weight and score gradient of one (query, key) pair ------------------
-// p = 2^(s c - lse log2 e) with the forward's log-sum-exp; ds = (p (dp - delta)) scale.
+// p = 2^(s c - lse log2 e) with the forward's log-sum-exp; ds = p (dp - delta): the softmax scale
+// is applied once per output element when dQ / dK leave their fp32 accumulators.
 __device__ __forceinline__ float bwd_p(float s, float c, float lse_log2) { return ex2_ftz(__fmaf_rn(s, c, -lse_log2)); }
-__device__ __forceinline__ float bwd_ds(float p, float dp, float delta, float scale) {
-    return __fmul_rn(__fmul_rn(p, __fsub_rn(dp, delta)), scale);
+__device__ __forceinline__ float bwd_ds(float p, float dp, float delta) { return __fmul_rn(p, __fsub_rn(dp, delta)); }
+// the same for two neighbouring columns with two-wide instructions (identical roundings)
+__device__ __forceinline__ void bwd_pds_x2(float s0, float s1, float dp0, float dp1, float c, float nl2_0, float nl2_1,
+                                           float ndl0, float ndl1, float& p0, float& p1, float& ds0, float& ds1) {
+    float x0, x1, t0, t1;
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %6};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(x0), "=f"(x1)
+        : "f"(s0), "f"(s1), "f"(c), "f"(nl2_0), "f"(nl2_1));
+    p0 = ex2_ftz(x0);
+    p1 = ex2_ftz(x1);
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(t0), "=f"(t1)
+        : "f"(dp0), "f"(dp1), "f"(ndl0), "f"(ndl1));
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(ds0), "=f"(ds1)
+        : "f"(p0), "f"(p1), "f"(t0), "f"(t1));
 }
 
 }  // namespace tik
