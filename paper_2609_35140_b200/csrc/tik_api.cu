@@ -497,7 +497,8 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     uint64_t bd[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(N)};
     uint64_t st1[1] = {static_cast<uint64_t>(K) * 2};
     uint32_t box[2] = {64, 128};
-    uint32_t boxB[2] = {64, 256};
+    const bool pair = T > 128;           // CTA pairs (two-SM MMAs) as soon as there is more than one row tile
+    uint32_t boxB[2] = {64, pair ? 128u : 256u};
     CUtensorMap tmY;
     uint64_t yd[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(T)};
     uint64_t ys[1] = {static_cast<uint64_t>(N) * 2};
@@ -518,7 +519,7 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     while (p.super_cols > 256 && ntile * ((N + p.super_cols - 1) / p.super_cols) < 4ll * ctx->sm_count) p.super_cols /= 2;
     p.nsuper = (N + p.super_cols - 1) / p.super_cols;
     p.dev_status = ctx->dev_status;
-    cudaError_t e = launch_linear(tmA, tmB, tmY, p, static_cast<cudaStream_t>(stream));
+    cudaError_t e = launch_linear(tmA, tmB, tmY, p, pair, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_linear");
 }
 

@@ -118,7 +118,7 @@ struct LinearParams {
     int* dev_status;
 };
 cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
-                          const LinearParams& p, cudaStream_t stream);
+                          const LinearParams& p, bool pair, cudaStream_t stream);
 
 struct BwdParams {
     const int32_t* cu_seqlens;   // [S+1]

@@ -14,27 +14,37 @@
 namespace tik {
 
 namespace lin {
-constexpr int STAGES = 4;
 constexpr int NB = 256;                      // output columns per MMA
 constexpr uint32_t A_BYTES = 128 * 128;      // 128 rows x 64 bf16
-constexpr uint32_t B_BYTES = NB * 128;       // 256 W rows x 64 bf16
-constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr uint32_t STG_BYTES = 128 * 128;    // output staging: 128 rows x 64 bf16, two buffers
-constexpr uint32_t OFF_STG = STAGES * STAGE_BYTES;
-constexpr uint32_t OFF_BAR = OFF_STG + 2 * STG_BYTES;
-constexpr uint32_t BYTES = OFF_BAR + 256;
-constexpr uint32_t ALLOC = BYTES + 1024;
-constexpr int BAND = 32;                     // row tiles per L2 band
+constexpr int BAND = 32;                     // row tiles per L2 band (even: CTA pairs stay inside a band)
 constexpr int THREADS = 192;                 // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+// PAIR: two CTAs on neighbouring SMs share every MMA (M = 256 rows); each stages its own 128 rows of
+// x and 128 of the 256 weight rows of a step, as in the log-probability kernel.
+template <bool PAIR>
+struct Cfg {
+    static constexpr int STAGES = PAIR ? 6 : 4;
+    static constexpr uint32_t B_BYTES = (PAIR ? NB / 2 : NB) * 128;
+    static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr uint32_t OFF_STG = STAGES * STAGE_BYTES;
+    static constexpr uint32_t OFF_BAR = OFF_STG + 2 * STG_BYTES;
+    static constexpr uint32_t BYTES = OFF_BAR + 256;
+    static constexpr uint32_t ALLOC = BYTES + 1024;
+};
 }  // namespace lin
 
+template <bool PAIR>
 __global__ void __launch_bounds__(lin::THREADS, 1)
 linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
               const __grid_constant__ CUtensorMap tmY, const LinearParams p) {
     using namespace lin;
+    using C = Cfg<PAIR>;
+    constexpr int STAGES = C::STAGES;
+    constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES, OFF_STG = C::OFF_STG, OFF_BAR = C::OFF_BAR;
     constexpr uint32_t TMEM_COLS = 512;      // two 256-column accumulators
-    constexpr uint32_t IDESC = mma_idesc_bf16(128, NB, false);
+    constexpr uint32_t IDESC = mma_idesc_bf16(PAIR ? 256 : 128, NB, false);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;     // 0 = the CTA that issues the pair's MMAs
 
     // raster: bands of BAND row tiles; within a band the row tile varies fastest so the CTAs in
     // flight share one super-chunk of W in L2 and W is streamed from HBM once per band
@@ -45,7 +55,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const long long rem = blockIdx.x - band * per_band;
     const int sup = static_cast<int>(rem / BAND);
     const int tile_in_band = static_cast<int>(rem % BAND);
-    if (tile_in_band >= band_tiles) return;
+    if ((PAIR ? (tile_in_band & ~1) : tile_in_band) >= band_tiles) return;   // a pair leaves only together
     const int row0 = (band * BAND + tile_in_band) * 128;
     const int col_base = sup * p.super_cols;
     const int n_nt = min(p.super_cols / NB, (p.N - col_base + NB - 1) / NB);   // 256-column steps
@@ -70,7 +80,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
-            mbar_init(bar_acc_empty + 8 * b, 128);
+            mbar_init(bar_acc_empty + 8 * b, PAIR ? 256 : 128);
         }
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
         fence_barrier_init();
@@ -79,13 +89,23 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         tma_prefetch_desc(&tmY);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
-        tmem_relinquish();
+        if (PAIR) {
+            tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();            // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    const uint32_t lead_full = PAIR ? mapa_cluster(bar_full, 0) : bar_full;
+    const uint32_t lead_acc_empty = PAIR ? mapa_cluster(bar_acc_empty, 0) : bar_acc_empty;
+    const uint32_t peer_empty = PAIR ? mapa_cluster(bar_empty, 1) : bar_empty;
+    const uint32_t peer_acc_full = PAIR ? mapa_cluster(bar_acc_full, 1) : bar_acc_full;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -98,16 +118,23 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     const int s = it % STAGES;
                     const uint32_t use = it / STAGES;
                     if (use > 0) mbar_wait(bar_empty + 8 * s, (use - 1) & 1, abort_word, p.dev_status);
-                    mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
                     // rows past T and W rows past N are outside the tensor maps and arrive as zeros
-                    tma_load_2d(sbase + s * STAGE_BYTES, &tmA, bar_full + 8 * s, kb * 64, row0);
-                    tma_load_2d(sbase + s * STAGE_BYTES + A_BYTES, &tmB, bar_full + 8 * s, kb * 64, col0);
+                    if (PAIR) {
+                        if (rank == 0) mbar_expect_tx(bar_full + 8 * s, 2 * STAGE_BYTES);   // both CTAs' bytes
+                        tma_load_2d_pair(sbase + s * STAGE_BYTES, &tmA, lead_full + 8 * s, kb * 64, row0);
+                        tma_load_2d_pair(sbase + s * STAGE_BYTES + A_BYTES, &tmB, lead_full + 8 * s, kb * 64,
+                                         col0 + 128 * static_cast<int>(rank));
+                    } else {
+                        mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
+                        tma_load_2d(sbase + s * STAGE_BYTES, &tmA, bar_full + 8 * s, kb * 64, row0);
+                        tma_load_2d(sbase + s * STAGE_BYTES + A_BYTES, &tmB, bar_full + 8 * s, kb * 64, col0);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             uint32_t it = 0;
             for (int nt = 0; nt < n_nt; ++nt) {
                 const int buf = nt & 1;
@@ -120,11 +147,23 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     mbar_wait(bar_full + 8 * s, (it / STAGES) & 1, abort_word, p.dev_status);
                     tc_fence_after();
                     const uint32_t a0 = sbase + s * STAGE_BYTES, b0 = a0 + A_BYTES;
-                    mma_ss_chain4(tmem + buf * NB, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
-                                  IDESC, kb ? 1u : 0u);
-                    mma_commit(bar_empty + 8 * s);
+                    if (PAIR) {
+                        mma_ss_chain4_pair(tmem + buf * NB, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
+                                           IDESC, kb ? 1u : 0u);
+                        mma_commit_pair(bar_empty + 8 * s);
+                        mma_commit_pair(peer_empty + 8 * s);
+                    } else {
+                        mma_ss_chain4(tmem + buf * NB, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
+                                      IDESC, kb ? 1u : 0u);
+                        mma_commit(bar_empty + 8 * s);
+                    }
                 }
-                mma_commit(bar_acc_full + 8 * buf);
+                if (PAIR) {
+                    mma_commit_pair(bar_acc_full + 8 * buf);
+                    mma_commit_pair(peer_acc_full + 8 * buf);
+                } else {
+                    mma_commit(bar_acc_full + 8 * buf);
+                }
             }
         }
     } else {
@@ -172,7 +211,8 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             }
             // all TMEM reads of this accumulator are done: hand it back to the MMA warp
             tc_fence_before();
-            mbar_arrive(bar_acc_empty + 8 * buf);
+            if (PAIR) mbar_arrive_cluster(lead_acc_empty + 8 * buf);
+            else mbar_arrive(bar_acc_empty + 8 * buf);
         }
         if (warp == 2 && lane == 0) tma_store_wait_read();     // shared memory stays valid until the last read
     }
@@ -184,24 +224,48 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
+    if (PAIR) cluster_sync_all();            // neither CTA leaves while the other may still touch it
+    if (warp == 1) {
+        if (PAIR) tmem_dealloc_pair(tmem, TMEM_COLS);
+        else tmem_dealloc(tmem, TMEM_COLS);
+    }
 }
 
-cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
-                          const LinearParams& p, cudaStream_t stream) {
-    if (p.T <= 0) return cudaSuccess;
+template <bool PAIR>
+static cudaError_t launch_linear_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                                   const LinearParams& p, cudaStream_t stream) {
+    using C = lin::Cfg<PAIR>;
+    auto kern = linear_kernel<PAIR>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(lin::ALLOC));
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(C::ALLOC));
         if (e != cudaSuccess) return e;
         configured = true;
     }
     const long long ntile = (p.T + 127) / 128;
     const long long nband = (ntile + lin::BAND - 1) / lin::BAND;
-    const long long grid = nband * lin::BAND * p.nsuper;
-    linear_kernel<<<static_cast<unsigned>(grid), lin::THREADS, lin::ALLOC, stream>>>(tmA, tmB, tmY, p);
-    return cudaGetLastError();
+    const long long grid = nband * lin::BAND * p.nsuper;         // even: BAND is
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(lin::THREADS);
+    cfg.dynamicSmemBytes = C::ALLOC;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
+}
+
+// pair = true: tmB must have a box of 128 rows (each CTA of a pair stages half of a step's 256)
+cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                          const LinearParams& p, bool pair, cudaStream_t stream) {
+    if (p.T <= 0) return cudaSuccess;
+    return pair ? launch_linear_t<true>(tmA, tmB, tmY, p, stream) : launch_linear_t<false>(tmA, tmB, tmY, p, stream);
 }
 
 }  // namespace tik
