@@ -365,7 +365,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-
     auto chunk_of = [&](int it) { return (tile_first + it) / TILES_PER_CHUNK; };
     auto is_chunk_start = [&](int it) { return ((tile_first + it) % TILES_PER_CHUNK) == 0; };
     auto col_o_of = [&](int it) -> uint32_t {
@@ -375,6 +374,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         return chunk_of(it) == 0 ? COL_OA : COL_OB;
     };
 
+    // Register budget: the four role warps (one warpgroup) need few registers, a softmax thread
+    // holds a 128-column score row.  128 x 88 + 256 x 208 = 64 512 registers.
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     if (warp == 0 || warp == 2) {
         // ------------------------------------------------------------ TMA producers
         // warp 0 streams Q and the K tiles, warp 2 the V tiles: a K tile is requested as soon as
@@ -455,7 +458,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             }
         }
         __syncwarp();
-    } else if (warp >= 4) {
+    }
+    } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+    {
         // ------------------------------------------------------------ softmax (two warpgroups)
         // The warpgroups alternate over KV tiles: warpgroup wg owns the tiles with it % 2 == wg
         // and with them score buffer wg, one thread per row and all 128 columns of the tile.
@@ -941,6 +947,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             }
         }
         }
+    }
     }
 
     // ---------------------------------------------------------------- teardown
