@@ -321,38 +321,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // an earlier kernel on this context may have run out of a wait: then do nothing at all
         if (lane == 0)
             *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
-        // Query tiles are read once, so a CTA's first load is a DRAM miss of ~1.5 us with nothing
-        // to overlap it.  CTAs start roughly in block order as SMs free up: prefetch into L2 the
-        // query tiles of the CTA that comes `lookahead` blocks later, which starts about when this
-        // one ends.
-        if (MODE != MODE_DECODE && lane == 0) {
-            const long long nblk = static_cast<long long>(gridDim.x) * gridDim.y * gridDim.z;
-            const long long lin = (static_cast<long long>(blockIdx.z) * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
-            const long long nxt = lin + p.lookahead;
-            if (nxt < nblk) {
-                const int bx = static_cast<int>(nxt % gridDim.x);
-                const int by = static_cast<int>((nxt / gridDim.x) % gridDim.y);
-                const int bz = static_cast<int>(nxt / (static_cast<long long>(gridDim.x) * gridDim.y));
-                int qb2 = p.cu_seqlens[bz], ctx2, pos2;
-                if (MODE == MODE_TRAIN) {
-                    ctx2 = p.cu_seqlens[bz + 1] - qb2;
-                    pos2 = 0;
-                } else {
-                    ctx2 = p.ctx_lens[bz];
-                    pos2 = ctx2 - (p.cu_seqlens[bz + 1] - qb2);
-                }
-                if (ctx2 > 0 && pos2 >= 0) {
-                    const int x2 = gridDim.x - 1 - bx;
-                    const int t_lo2 = pos2 / 128, t_hi2 = (ctx2 - 1) / 128;
-                    for (int q2 = 0; q2 < 2; ++q2) {
-                        const int Tq = (x2 >= 8) ? (16 + x2 - 8) : (2 * x2 + q2);
-                        if ((x2 >= 8 && q2 == 1) || Tq < t_lo2 || Tq > t_hi2) continue;
-                        const int row = qb2 + 128 * Tq - pos2;
-                        for (int a = 0; a < NATOM; ++a) tma_prefetch_l2_3d(&tmQ, a * 64, by, row);
-                    }
-                }
-            }
-        }
     }
     if (MODE == MODE_DECODE) {
         // rows >= G of the Q tile are never loaded: zero them (their scores and weights stay 0)
@@ -440,6 +408,40 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         __syncwarp();
     } else if (warp == 3) {
         // ------------------------------------------------------------ PV issuer
+        // (done here, after the set-up synchronisation: its dependent global loads would otherwise
+        // hold up every warp of the CTA, and this thread has nothing to do until the first weights)
+        // Query tiles are read once, so a CTA's first load is a DRAM miss of ~1.5 us with nothing
+        // to overlap it.  CTAs start roughly in block order as SMs free up: prefetch into L2 the
+        // query tiles of the CTA that comes `lookahead` blocks later, which starts about when this
+        // one ends.
+        if (MODE != MODE_DECODE && lane == 0) {
+            const long long nblk = static_cast<long long>(gridDim.x) * gridDim.y * gridDim.z;
+            const long long lin = (static_cast<long long>(blockIdx.z) * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+            const long long nxt = lin + p.lookahead;
+            if (nxt < nblk) {
+                const int bx = static_cast<int>(nxt % gridDim.x);
+                const int by = static_cast<int>((nxt / gridDim.x) % gridDim.y);
+                const int bz = static_cast<int>(nxt / (static_cast<long long>(gridDim.x) * gridDim.y));
+                int qb2 = p.cu_seqlens[bz], ctx2, pos2;
+                if (MODE == MODE_TRAIN) {
+                    ctx2 = p.cu_seqlens[bz + 1] - qb2;
+                    pos2 = 0;
+                } else {
+                    ctx2 = p.ctx_lens[bz];
+                    pos2 = ctx2 - (p.cu_seqlens[bz + 1] - qb2);
+                }
+                if (ctx2 > 0 && pos2 >= 0) {
+                    const int x2 = gridDim.x - 1 - bx;
+                    const int t_lo2 = pos2 / 128, t_hi2 = (ctx2 - 1) / 128;
+                    for (int q2 = 0; q2 < 2; ++q2) {
+                        const int Tq = (x2 >= 8) ? (16 + x2 - 8) : (2 * x2 + q2);
+                        if ((x2 >= 8 && q2 == 1) || Tq < t_lo2 || Tq > t_hi2) continue;
+                        const int row = qb2 + 128 * Tq - pos2;
+                        for (int a = 0; a < NATOM; ++a) tma_prefetch_l2_3d(&tmQ, a * 64, by, row);
+                    }
+                }
+            }
+        }
         if (lane == 0) {
             for (int g = 0; g < n_steps; ++g) {
                 const int vt = pair ? (g >> 1) : g;
@@ -745,37 +747,38 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             // buffer) and one tiled TMA store; a ragged tile is written row by row.
             const bool full_tile = e_lo == 0 && e_hi == 128;
             uint8_t* stage = smem + L::OFF_Q + wg * L::TILE;
+            // 64 columns (one swizzle atom) at a time: both TMEM loads of an atom are in flight
+            // together, and the atom's TMA store reads shared memory while the next one is staged
 #pragma unroll
-            for (int cc = 0; cc < D / 32; ++cc) {
-                uint32_t v[32];
-                tmem_ld32(to + 32 * cc, v);
+            for (int a = 0; a < NATOM; ++a) {
+                uint32_t v[64];
+                tmem_ld32(to + 64 * a, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                tmem_ld32(to + 64 * a + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
                 tmem_wait_ld();
-                uint32_t o16[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    o16[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv),
-                                         finalize_o(__uint_as_float(v[2 * i + 1]), inv));
+                for (int i = 0; i < 8; ++i) {                 // 16-byte chunks of the atom's 128-byte row
+                    uint32_t w4[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint4 val = make_uint4(o16[4 * i], o16[4 * i + 1], o16[4 * i + 2], o16[4 * i + 3]);
+                    for (int j = 0; j < 4; ++j)
+                        w4[j] = pack_bf16x2(finalize_o(__uint_as_float(v[8 * i + 2 * j]), inv),
+                                            finalize_o(__uint_as_float(v[8 * i + 2 * j + 1]), inv));
+                    const uint4 val = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                     if (full_tile) {
-                        const int c16 = 4 * cc + i;             // 16-byte chunk of the row
-                        *reinterpret_cast<uint4*>(stage + (c16 >> 3) * L::ATOM + r * 128 + (((c16 & 7) ^ (r & 7)) << 4)) = val;
+                        *reinterpret_cast<uint4*>(stage + a * L::ATOM + r * 128 + ((i ^ (r & 7)) << 4)) = val;
                     } else if (valid) {
-                        reinterpret_cast<uint4*>(optr + 32 * cc)[i] = val;
+                        reinterpret_cast<uint4*>(optr + 64 * a)[i] = val;
+                    }
+                }
+                if (full_tile) {
+                    fence_proxy_async_smem();
+                    named_bar_sync(2 + wg, 128);
+                    if (quarter == 0 && lane == 0) {
+                        tma_store_3d(&p.tmO, smem_u32(stage) + a * L::ATOM, a * 64, head, e_row0);
+                        tma_store_commit();
                     }
                 }
             }
-            if (full_tile) {
-                fence_proxy_async_smem();
-                named_bar_sync(2 + wg, 128);
-                if (quarter == 0 && lane == 0) {
-                    for (int a = 0; a < NATOM; ++a)
-                        tma_store_3d(&p.tmO, smem_u32(stage) + a * L::ATOM, a * 64, head, e_row0);
-                    tma_store_commit();
-                    tma_store_wait_read();
-                }
-            }
+            if (full_tile && quarter == 0 && lane == 0) tma_store_wait_read();
         } else {
         for (int it = wg; it < n_tiles; it += 2) {
             const int j = tile_first + it;
