@@ -393,8 +393,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const int st = (KS == 2) ? (kt & 1) : (kt % KV_STAGES), b = g & 1;
                 const int kuse = (KS == 2) ? (kt >> 1) : (kt / KV_STAGES);
                 // the single score buffer is free once the softmax of step g-1 holds it in registers
-                if (g >= 1) mbar_wait(bar_sempty + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_word, p.dev_status);
                 mbar_wait(bar_kfull + 8 * st, kuse & 1, abort_word, p.dev_status);
+                if (g >= 1) mbar_wait(bar_sempty + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_word, p.dev_status);
                 tc_fence_after();
                 const uint64_t dq = (pair && b) ? dq1 : dq0;
                 const uint64_t dk = smem_desc_sw128(sK + st * L::TILE, 0, 1024);
@@ -558,7 +558,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const bool chunk_start = is_chunk_start(it);
                 const bool fold_now = chunk_start && it > 0;      // a finished chunk precedes this tile
                 mbar_wait(bar_sfull + 8 * wg, (it >> 1) & 1, abort_word, p.dev_status);
-                if (it >= 2) wait_pv(it - 2);
                 tc_fence_after();
                 uint32_t sc[32];
                 tmem_ld32(ts + 32 * quarter, sc);
@@ -630,6 +629,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     uint32_t pk[64];
 #pragma unroll
                     for (int i = 0; i < 64; i += 8) softmax_sum_pack8(&x[i], rs_lo, &pk[i >> 1]);
+                    // the weight buffer of this warpgroup was last read by the PV of tile it-2
+                    if (it >= 2) wait_pv(it - 2);
                     tmem_st32(tp, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
 #pragma unroll
                     for (int i = 0; i < 64; i += 8) softmax_sum_pack8(&x[64 + i], rs_hi, &pk[32 + (i >> 1)]);
@@ -654,6 +655,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         rescale_o_tmem<D>(tlane + col_o_of(it), alpha);
                     }
                     tmem_wait_st();
+                } else if (it >= 2) {
+                    wait_pv(it - 2);     // every warp passes this wait before it arrives for tile it
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -681,8 +684,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 g_last = g;
                 const int j = g >> 1;
                 mbar_wait(bar_sfull + 8 * wg, (g >> 1) & 1, abort_word, p.dev_status);
-                // the PV of step g-2 read this warpgroup's weight buffer and updated its accumulator
-                if (g >= 2) wait_pv(g - 2);
                 tc_fence_after();
                 const int kmax = qpos_p - 128 * j;              // columns > kmax are masked
                 uint32_t sc[128];
@@ -719,6 +720,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 rs_hi.reset();
 #pragma unroll
                 for (int i = 0; i < 64; i += 8) softmax_p8(&sc[i], c, neg_mc, rs_lo, &sc[i >> 1]);
+                // The PV of step g-2 read this warpgroup's weight buffer and updated its
+                // accumulator.  It is waited for here, right before the first store: in front of
+                // the score load the same wait sat inside both the softmax chain and the
+                // load -> QK^T -> load cycle of the score buffer (measured: 7-9 % of the kernel).
+                if (g >= 2) wait_pv(g - 2);
                 tmem_st32(tp, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
 #pragma unroll
                 for (int i = 0; i < 64; i += 8) softmax_p8(&sc[64 + i], c, neg_mc, rs_hi, &sc[32 + (i >> 1)]);
@@ -784,11 +790,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             const int j = tile_first + it;
             const bool chunk_start = is_chunk_start(it);
             mbar_wait(bar_sfull + 8 * wg, (it >> 1) & 1, abort_word, p.dev_status);
-            // The weight buffer of this warpgroup was last read by the PV of tile it-2.  Every
-            // warp waits for it, idle ones too: it also keeps a warp from arriving for tile it on
-            // a barrier whose phase for tile it-2 is still collecting arrivals.
-            if (it >= 2) wait_pv(it - 2);
             tc_fence_after();
+            if (!active && it >= 2) wait_pv(it - 2);
             if (active) {
                 const int kmax = qpos - 128 * j;            // columns > kmax are masked
                 uint32_t sc[128];
@@ -843,6 +846,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 // a masked score is -inf: the fma gives -inf and ex2 gives +0 exactly
 #pragma unroll
                 for (int i = 0; i < 64; i += 8) softmax_p8(&sc[i], c, neg_mc, rs_lo, &sc[i >> 1]);
+                // The weight buffer of this warpgroup was last read by the PV of tile it-2: waited
+                // for right before the first store, not in front of the score load.  Every warp
+                // passes this wait before it arrives for tile it, so no arrival can land in the
+                // barrier phase of tile it-2.
+                if (it >= 2) wait_pv(it - 2);
                 tmem_st32(tp, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
 #pragma unroll
                 for (int i = 0; i < 64; i += 8) softmax_p8(&sc[64 + i], c, neg_mc, rs_hi, &sc[32 + (i >> 1)]);
