@@ -476,8 +476,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         const int quarter = warp & 3;                       // TMEM lane quarter of this warp
         const int r = quarter * 32 + lane;                  // tile row == TMEM lane
         const uint32_t tlane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
-        const int qpos = (MODE == MODE_DECODE) ? (ctx - 1) : (128 * T0 + r);
-        const bool active = (MODE != MODE_DECODE) || (quarter == 0);
+        const int qpos = 128 * T0 + r;      // train / prefill, single mode: position of this thread's row
         const float c = p.c;
         float* st_m = lx;                 // [128]    running maximum of the current chunk
         float* st_l = lx + 128;           // [2][128] half row sums of the current chunk
@@ -791,8 +790,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             const bool chunk_start = is_chunk_start(it);
             mbar_wait(bar_sfull + 8 * wg, (it >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
-            if (!active && it >= 2) wait_pv(it - 2);
-            if (active) {
+            {
                 const int kmax = qpos - 128 * j;            // columns > kmax are masked
                 uint32_t sc[128];
                 tmem_ld32(ts, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
@@ -869,12 +867,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 st_l[128 + r] = l_own_hi;
                 if (fold_now) {
                     wait_pv(it - 1);
-                    if (MODE == MODE_DECODE) {
-                        write_partial_ml(chunk_of(it - 1), m_prev, l_prev_lo, l_prev_hi);
-                        write_partial_o(chunk_of(it - 1), 0, D);
-                    } else {
-                        fold_chunk(chunk_of(it - 1), m_prev, l_prev_lo, l_prev_hi, true);
-                    }
+                    fold_chunk(chunk_of(it - 1), m_prev, l_prev_lo, l_prev_hi, true);
                 } else if (!chunk_start && !__all_sync(0xffffffffu, alpha == 1.0f)) {
                     // rescale the chunk accumulator of this row
                     wait_pv(it - 1);
@@ -882,40 +875,29 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
                 tmem_wait_st();
                 // this thread closed a chunk that is not the row's last: fold its scalars here too
-                if (MODE != MODE_DECODE && it != last && ((tile_first + it) % TILES_PER_CHUNK) == TILES_PER_CHUNK - 1)
+                if (it != last && ((tile_first + it) % TILES_PER_CHUNK) == TILES_PER_CHUNK - 1)
                     fold_chunk(chunk_of(it), m_own, l_own_lo, l_own_hi, false);
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) {
-                if (!active) mbar_arrive(bar_sempty + 8 * wg);
-                mbar_arrive(bar_pfull + 8 * wg);
-            }
+            if (lane == 0) mbar_arrive(bar_pfull + 8 * wg);
         }
 
         // ---- the warpgroup that owned the last tile finishes the row state
         if (wg == (last & 1)) {
             wait_pv(last);
-            if (active) {
-                if (MODE == MODE_DECODE) {
-                    write_partial_ml(chunk_of(last), m_own, l_own_lo, l_own_hi);
-                } else {
-                    fold_chunk(chunk_of(last), m_own, l_own_lo, l_own_hi, true);
-                    const float Ltot = finalize_l(Lg_lo, Lg_hi);
-                    st_m[r] = finalize_inv(Ltot);       // the hand-off slots are free now
-                    const bool valid = (r >= meta[1]) && (r < meta[2]);
-                    if (valid && p.lse) p.lse[(static_cast<long long>(meta[0]) + r) * p.Hq + head] = finalize_lse(M_g, Ltot, c);
-                }
-            }
+            fold_chunk(chunk_of(last), m_own, l_own_lo, l_own_hi, true);
+            const float Ltot = finalize_l(Lg_lo, Lg_hi);
+            st_m[r] = finalize_inv(Ltot);       // the hand-off slots are free now
+            const bool valid = (r >= meta[1]) && (r < meta[2]);
+            if (valid && p.lse) p.lse[(static_cast<long long>(meta[0]) + r) * p.Hq + head] = finalize_lse(M_g, Ltot, c);
             tc_fence_before();
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         tc_fence_after();
         // both warpgroups write half of the output columns each
-        if (active) {
-            if (MODE == MODE_DECODE) {
-                write_partial_o(chunk_of(last), DH * wg, DH);
-            } else {
+        {
+            {
                 const float inv = st_m[r];
                 const int e_row0 = meta[0], e_lo = meta[1], e_hi = meta[2];
                 const bool valid = (r >= e_lo) && (r < e_hi);
