@@ -35,7 +35,7 @@ struct BwdSmem {
     static constexpr uint32_t OFF_R = 0;                  // two resident row-side tiles
     static constexpr uint32_t OFF_C = 2 * TILE;           // BWD_STAGES x two streamed tiles
     static constexpr uint32_t OFF_BAR = OFF_C + BWD_STAGES * 2 * TILE;
-    static constexpr uint32_t OFF_SC = OFF_BAR + 128;     // [half][buffer][l2 | delta][64] floats of the columns
+    static constexpr uint32_t OFF_SC = OFF_BAR + 128;     // [half][buffer][-l2 x 64 | -delta x 64] floats of the columns
     static constexpr uint32_t BYTES = OFF_SC + 2 * 2 * 2 * 64 * 4;
     static constexpr uint32_t ALLOC = BYTES + 1024;       // slack to align the base to 1 KiB
 };
@@ -223,7 +223,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // DKV: the scalars belong to the columns (query rows of the streamed tile).  Thread `et` < 64
         // of warpgroup h fetches those of column 64 h + et one step ahead; they reach the other
         // threads of the warpgroup through shared memory (double-buffered, one named barrier per step).
-        float* my_sc = sc_base + hlf * (2 * 2 * 64);          // [buffer][64][l2, delta]
+        // (stored negated and as two arrays, so that two neighbouring columns' values load as one
+        // 8-byte pair, ready for the two-wide arithmetic)
+        float* my_sc = sc_base + hlf * (2 * 2 * 64);          // [buffer][-l2 x 64 | -delta x 64]
         auto fetch_col = [&](int t, float& l2, float& dl) {
             l2 = 0.0f;
             dl = 0.0f;
@@ -240,15 +242,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             float l2, dl;
             fetch_col(0, l2, dl);
             if (et < 64) {
-                my_sc[2 * et] = l2;
-                my_sc[2 * et + 1] = dl;
+                my_sc[et] = -l2;
+                my_sc[64 + et] = -dl;
             }
             named_bar_sync(1 + hlf, 256);
         }
         for (int t = 0; t < n_steps; ++t) {
             float nl2 = 0.0f, ndl = 0.0f;
             if (MODE == BWD_DKV) fetch_col(t + 1, nl2, ndl);            // in flight during this step
-            const float2* csc = reinterpret_cast<const float2*>(my_sc + (t & 1) * 128);   // (l2, delta) per column
+            const float* csc = my_sc + (t & 1) * 128 + 32 * sub;       // -l2 of this thread's 32 columns; -delta at + 64
             mbar_wait(bar_tfull + 8 * hlf, t & 1, abort_word, p.dev_status);
             tc_fence_after();
             // column cc of the half is masked for this row when it lies in the row's future (DQ: key
@@ -274,8 +276,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                             nl2_0 = nl2_1 = -row_l2;
                             ndl0 = ndl1 = -row_dl;
                         } else {
-                            const float4 sc4 = *reinterpret_cast<const float4*>(&csc[32 * sub + i]);   // (l2, dl) x 2
-                            nl2_0 = -sc4.x, ndl0 = -sc4.y, nl2_1 = -sc4.z, ndl1 = -sc4.w;
+                            const float2 nl = *reinterpret_cast<const float2*>(&csc[i]);
+                            const float2 nd = *reinterpret_cast<const float2*>(&csc[64 + i]);
+                            nl2_0 = nl.x, nl2_1 = nl.y, ndl0 = nd.x, ndl1 = nd.y;
                         }
                         float p0, p1, ds0, ds1;
                         bwd_pds_x2(__uint_as_float(s_[i]), __uint_as_float(s_[i + 1]), __uint_as_float(d_[i]),
@@ -299,9 +302,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                                 dl = row_dl;
                             } else {
                                 masked = (row_abs > col_abs) || (col_abs >= len);
-                                const float2 sc2 = csc[32 * sub + cc];
-                                l2 = sc2.x;
-                                dl = sc2.y;
+                                l2 = -csc[cc];
+                                dl = -csc[64 + cc];
                             }
                             const float pe = bwd_p(__uint_as_float(s_[i + e]), c, l2);
                             pv[e] = masked ? 0.0f : pe;
@@ -319,8 +321,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 // hand the next step's column scalars over (the buffer was last read a step ago, before
                 // the previous barrier)
                 if (et < 64) {
-                    my_sc[((t + 1) & 1) * 128 + 2 * et] = nl2;
-                    my_sc[((t + 1) & 1) * 128 + 2 * et + 1] = ndl;
+                    my_sc[((t + 1) & 1) * 128 + et] = -nl2;
+                    my_sc[((t + 1) & 1) * 128 + 64 + et] = -ndl;
                 }
                 named_bar_sync(1 + hlf, 256);
             }
