@@ -28,28 +28,37 @@ enum { BWD_DQ = 0, BWD_DKV = 1 };
 constexpr int BWD_THREADS = 576;     // warp 0 TMA, warp 1 MMA, warps 2-17 element-wise (four threads per tile row)
 constexpr int BWD_STAGES = 2;
 
-template <int D>
+template <int D, int MODE>
 struct BwdSmem {
     static constexpr uint32_t ATOM = 128 * 128;           // 128 rows x 64 bf16
     static constexpr uint32_t TILE = (D / 64) * ATOM;
     static constexpr uint32_t OFF_R = 0;                  // two resident row-side tiles
-    static constexpr uint32_t OFF_C = 2 * TILE;           // BWD_STAGES x two streamed tiles
-    static constexpr uint32_t OFF_BAR = OFF_C + BWD_STAGES * 2 * TILE;
-    static constexpr uint32_t OFF_SC = OFF_BAR + 128;     // [half][buffer][-l2 x 64 | -delta x 64] floats of the columns
-    static constexpr uint32_t BYTES = OFF_SC + 2 * 2 * 2 * 64 * 4;
+    // streamed tiles.  DKV: BWD_STAGES stages of (Q_i, dO_i).  DQ: three K stages, then two V
+    // stages (a V tile is done with after its dP product, a K tile only after the gradient product).
+    static constexpr uint32_t OFF_C = 2 * TILE;
+    static constexpr uint32_t N_STREAM = (MODE == 0) ? 5 : 2 * BWD_STAGES;
+    static constexpr uint32_t OFF_BAR = OFF_C + N_STREAM * TILE;
+    static constexpr uint32_t OFF_SC = OFF_BAR + 144;     // DKV: [half][buffer][-l2 x 64 | -delta x 64] floats of the columns
+    static constexpr uint32_t BYTES = OFF_SC + ((MODE == 0) ? 0 : 2 * 2 * 2 * 64 * 4);
     static constexpr uint32_t ALLOC = BYTES + 1024;       // slack to align the base to 1 KiB
 };
+constexpr int DQ_KSTAGES = 3, DQ_VSTAGES = 2;
 
 template <int D, int MODE>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
                 const BwdParams p) {
-    using L = BwdSmem<D>;
+    using L = BwdSmem<D, MODE>;
     constexpr int NATOM = D / 64;
     constexpr uint32_t TMEM_COLS = 512;
-    constexpr uint32_t COL_T1 = 0, COL_T2 = 128, COL_A1 = 256, COL_A2 = 256 + D;
+    // TMEM columns.  DKV: two score tiles (weights in place), two accumulators.  DQ: the score tile
+    // S, two dP tiles used alternately (dS in place), one accumulator.
+    constexpr uint32_t COL_T1 = 0, COL_T2 = 128;
+    constexpr uint32_t COL_T2B = 256;                                   // DQ only
+    constexpr uint32_t COL_A1 = (MODE == BWD_DQ) ? 384 : 256, COL_A2 = 256 + D;
     constexpr uint32_t IDESC_SC = mma_idesc_bf16(128, 64, false);       // one half: 64 streamed rows
+    constexpr uint32_t IDESC_SC128 = mma_idesc_bf16(128, 128, false);   // DQ: all 128 streamed rows at once
     constexpr uint32_t IDESC_OUT = mma_idesc_bf16(128, D, true);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -84,24 +93,32 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t sR1 = sbase + L::OFF_R, sR2 = sR1 + L::TILE;
     const uint32_t bar0 = sbase + L::OFF_BAR;
     const uint32_t bar_r = bar0;                 // row-side tiles landed
-    const uint32_t bar_cfull = bar0 + 8;         // [2] streamed tiles landed
-    const uint32_t bar_cempty = bar0 + 24;       // [2] gradient MMAs that read the stage are done
-    const uint32_t bar_tfull = bar0 + 40;        // [2] score MMAs of a half-step done
-    const uint32_t bar_efull = bar0 + 56;        // [2] weights of a half-step written to TMEM (4 warps)
-    const uint32_t bar_acc = bar0 + 72;          // all MMAs done
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 80);
-    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 84);
+    const uint32_t bar_cfull = bar0 + 8;         // [3] streamed tiles landed (DQ: K tiles)
+    const uint32_t bar_cempty = bar0 + 32;       // [3] gradient MMAs that read the stage are done
+    const uint32_t bar_vfull = bar0 + 56;        // [2] DQ: V tile landed
+    const uint32_t bar_vempty = bar0 + 72;       // [2] DQ: the dP product that read the V stage is done
+    const uint32_t bar_tfull = bar0 + 88;        // [2] score MMAs of a half-step done (DQ: [0] of a step,
+                                                 //     [1] "score tile S is in registers", 16 warps)
+    const uint32_t bar_efull = bar0 + 104;       // [2] weights of a half-step written to TMEM (8 warps; DQ:
+                                                 //     [0] dS of a step written, 16 warps)
+    const uint32_t bar_acc = bar0 + 120;         // all MMAs done
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 128);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 132);
     float* sc_base = reinterpret_cast<float*>(smem + L::OFF_SC);
 
     if (tid == 0) {
         mbar_init(bar_r, 1);
-        for (int i = 0; i < BWD_STAGES; ++i) {
+        for (int i = 0; i < 3; ++i) {
             mbar_init(bar_cfull + 8 * i, 1);
             mbar_init(bar_cempty + 8 * i, 1);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_tfull + 8 * i, 1);
-            mbar_init(bar_efull + 8 * i, 8);
+            mbar_init(bar_vfull + 8 * i, 1);
+            mbar_init(bar_vempty + 8 * i, 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_tfull + 8 * i, (MODE == BWD_DQ && i == 1) ? 16 : 1);
+            mbar_init(bar_efull + 8 * i, MODE == BWD_DQ ? 16 : 8);
         }
         mbar_init(bar_acc, 1);
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
@@ -134,6 +151,23 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     tma_load_3d(sR2 + a * L::ATOM, &tmV, bar_r, a * 64, kvh, row_own);
                 }
             }
+            if (MODE == BWD_DQ) {
+                for (int t = 0; t < n_steps; ++t) {
+                    if (*abort_word) break;          // a wait expired somewhere: stop issuing copies
+                    const int row = tok0 + 128 * t;
+                    const int ks = t % DQ_KSTAGES, vs = t % DQ_VSTAGES;
+                    const uint32_t kuse = t / DQ_KSTAGES, vuse = t / DQ_VSTAGES;
+                    if (kuse > 0) mbar_wait(bar_cempty + 8 * ks, (kuse - 1) & 1, abort_word, p.dev_status);
+                    mbar_expect_tx(bar_cfull + 8 * ks, L::TILE);
+                    for (int a = 0; a < NATOM; ++a)
+                        tma_load_3d(sbase + L::OFF_C + ks * L::TILE + a * L::ATOM, &tmK, bar_cfull + 8 * ks, a * 64, kvh, row);
+                    if (vuse > 0) mbar_wait(bar_vempty + 8 * vs, (vuse - 1) & 1, abort_word, p.dev_status);
+                    mbar_expect_tx(bar_vfull + 8 * vs, L::TILE);
+                    for (int a = 0; a < NATOM; ++a)
+                        tma_load_3d(sbase + L::OFF_C + (DQ_KSTAGES + vs) * L::TILE + a * L::ATOM, &tmV, bar_vfull + 8 * vs,
+                                    a * 64, kvh, row);
+                }
+            } else
             for (int t = 0; t < n_steps; ++t) {
                 if (*abort_word) break;          // a wait expired somewhere: stop issuing copies
                 const int st = t % BWD_STAGES;
@@ -184,6 +218,45 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     mma_ts_chain4(tmem + COL_A2, tmem + COL_T1 + 64 * h, smem_desc_sw128(c2, L::ATOM, 1024), IDESC_OUT,
                                   acc);
             };
+            if (MODE == BWD_DQ) {
+                // DQ: only dS feeds a gradient product, so the score tile S is free again as soon as
+                // the element-wise threads hold it in registers, and dP / dS alternate between two
+                // tiles.  Both score products of step t+1 (128 streamed rows each, which an SS-form
+                // MMA reads at the full rate; 64-row halves are bound by shared-memory bandwidth) are
+                // issued while the element-wise work of step t runs, the gradient product of step t
+                // right behind them.
+                auto stage_k = [&](int t) { return sbase + L::OFF_C + (t % DQ_KSTAGES) * L::TILE; };
+                auto score_full = [&](int t) {
+                    const uint32_t c1 = stage_k(t), c2 = sbase + L::OFF_C + (DQ_KSTAGES + t % DQ_VSTAGES) * L::TILE;
+                    const uint32_t t2 = tmem + ((t & 1) ? COL_T2B : COL_T2);
+                    mbar_wait(bar_cfull + 8 * (t % DQ_KSTAGES), (t / DQ_KSTAGES) & 1, abort_word, p.dev_status);
+                    mbar_wait(bar_vfull + 8 * (t % DQ_VSTAGES), (t / DQ_VSTAGES) & 1, abort_word, p.dev_status);
+                    if (t > 0) mbar_wait(bar_tfull + 8, (t - 1) & 1, abort_word, p.dev_status);   // S of step t-1 is in registers
+                    tc_fence_after();
+                    if (D == 128) {
+                        mma_ss_chain8_fresh(tmem + COL_T1, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC128);
+                        mma_ss_chain8_fresh(t2, dr2, smem_desc_sw128(c2, 0, 1024), IDESC_SC128);
+                    } else {
+                        mma_ss_chain4_fresh(tmem + COL_T1, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC128);
+                        mma_ss_chain4_fresh(t2, dr2, smem_desc_sw128(c2, 0, 1024), IDESC_SC128);
+                    }
+                    mma_commit(bar_tfull);
+                    mma_commit(bar_vempty + 8 * (t % DQ_VSTAGES));      // the V stage is done with
+                };
+                score_full(0);
+                for (int t = 0; t < n_steps; ++t) {
+                    if (*abort_word) break;
+                    if (t + 1 < n_steps) score_full(t + 1);
+                    mbar_wait(bar_efull, t & 1, abort_word, p.dev_status);
+                    tc_fence_after();
+                    // A = dS: every thread left its 32 columns' bf16 pairs in the first 16 columns of
+                    // its own 32-column block, so the eight 16-key steps sit at 0, 8, 32, 40, ...
+                    mma_ts_chain8_blocks(tmem + COL_A1, tmem + ((t & 1) ? COL_T2B : COL_T2),
+                                         smem_desc_sw128(stage_k(t), L::ATOM, 1024), IDESC_OUT, t > 0 ? 1u : 0u);
+                    mma_commit(bar_cempty + 8 * (t % DQ_KSTAGES));
+                }
+                mma_commit(bar_acc);
+            } else {
             mbar_wait(bar_cfull, 0, abort_word, p.dev_status);
             tc_fence_after();
             score(0, 0);
@@ -202,6 +275,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 }
             }
             mma_commit(bar_acc);
+            }
         }
         __syncwarp();
     } else {
@@ -247,6 +321,52 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             named_bar_sync(1 + hlf, 256);
         }
+        if (MODE == BWD_DQ) {
+            // DQ: all sixteen warps work on the same step, four threads per row with 32 columns each
+            const int cq = 2 * hlf + sub;
+            const float nl2 = -row_l2, ndl = -row_dl;
+            for (int t = 0; t < n_steps; ++t) {
+                mbar_wait(bar_tfull, t & 1, abort_word, p.dev_status);
+                tc_fence_after();
+                const uint32_t t2 = tlane + ((t & 1) ? COL_T2B : COL_T2) + 32 * cq;
+                uint32_t s_[32], d_[32];
+                tmem_ld32(tlane + COL_T1 + 32 * cq, s_);
+                tmem_ld32(t2, d_);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tfull + 8);      // S is in registers: the next QK^T may overwrite it
+                uint32_t dk_[16];
+                if (t != own) {               // off the diagonal nothing is masked: two-wide, no compares
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float p0, p1, ds0, ds1;
+                        bwd_pds_x2(__uint_as_float(s_[i]), __uint_as_float(s_[i + 1]), __uint_as_float(d_[i]),
+                                   __uint_as_float(d_[i + 1]), c, nl2, nl2, ndl, ndl, p0, p1, ds0, ds1);
+                        dk_[i >> 1] = pack_bf16x2(ds0, ds1);
+                    }
+                } else {
+                    const int col0_abs = 128 * t + 32 * cq;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float dsv[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const bool masked = col0_abs + i + e > row_abs;      // key after query
+                            const float pe = bwd_p(__uint_as_float(s_[i + e]), c, row_l2);
+                            dsv[e] = masked ? 0.0f : bwd_ds(pe, __uint_as_float(d_[i + e]), row_dl);
+                        }
+                        dk_[i >> 1] = pack_bf16x2(dsv[0], dsv[1]);
+                    }
+                }
+                // dS goes over the first 16 of this thread's own 32 dP columns: no other thread reads them
+                tmem_st16(t2, dk_);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_efull);
+            }
+        } else
         for (int t = 0; t < n_steps; ++t) {
             float nl2 = 0.0f, ndl = 0.0f;
             if (MODE == BWD_DKV) fetch_col(t + 1, nl2, ndl);            // in flight during this step
@@ -395,11 +515,11 @@ static cudaError_t launch_bwd_t(dim3 grid, const CUtensorMap& tmQ, const CUtenso
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(BwdSmem<D>::ALLOC));
+                                             static_cast<int>(BwdSmem<D, MODE>::ALLOC));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, BWD_THREADS, BwdSmem<D>::ALLOC, stream>>>(tmQ, tmK, tmV, tmDO, p);
+    kern<<<grid, BWD_THREADS, BwdSmem<D, MODE>::ALLOC, stream>>>(tmQ, tmK, tmV, tmDO, p);
     return cudaGetLastError();
 }
 

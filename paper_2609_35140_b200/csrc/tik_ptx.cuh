@@ -329,6 +329,22 @@ __device__ __forceinline__ void mma_ts_chain4(uint32_t d_tmem, uint32_t a_tmem, 
         : "memory");
 }
 
+// All eight steps with A laid out as four 32-column blocks whose first 16 columns hold the two
+// steps of that block (a thread that owns 32 fp32 columns of a tile leaves the bf16 pairs of its
+// 32 contraction rows in the first 16 of them).
+__device__ __forceinline__ void mma_ts_chain8_blocks(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                                     uint32_t idesc, uint32_t first_accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p0, pt;\n\t.reg .b64 db;\n\t.reg .b32 ta;\n\t"
+        "setp.ne.b32 p0, %4, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+        TIK_MMA_TS_STEP(8, 128) TIK_MMA_TS_STEP(32, 256) TIK_MMA_TS_STEP(40, 384)
+        TIK_MMA_TS_STEP(64, 512) TIK_MMA_TS_STEP(72, 640) TIK_MMA_TS_STEP(96, 768)
+        TIK_MMA_TS_STEP(104, 896)
+        "}" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(first_accumulate)
+        : "memory");
+}
+
 // ---------------------------------------------------------------- CTA pairs (cta_group::2)
 // Two CTAs of a cluster of two, on neighbouring SMs, execute one MMA of M = 256: each holds its
 // own 128 rows of A and half of the B tile in its shared memory and its own 128 accumulator rows
