@@ -25,7 +25,9 @@
 namespace tik {
 
 enum { BWD_DQ = 0, BWD_DKV = 1 };
-constexpr int BWD_THREADS = 576;     // warp 0 TMA, warp 1 MMA, warps 2-17 element-wise (four threads per tile row)
+// warp 0 TMA, warp 1 MMA (DQ: the score products), warps 2-17 element-wise (four threads per tile
+// row), warp 18 DQ: the gradient products
+constexpr int BWD_THREADS = 608;
 constexpr int BWD_STAGES = 2;
 
 template <int D, int MODE>
@@ -38,7 +40,7 @@ struct BwdSmem {
     static constexpr uint32_t OFF_C = 2 * TILE;
     static constexpr uint32_t N_STREAM = (MODE == 0) ? 5 : 2 * BWD_STAGES;
     static constexpr uint32_t OFF_BAR = OFF_C + N_STREAM * TILE;
-    static constexpr uint32_t OFF_SC = OFF_BAR + 144;     // DKV: [half][buffer][-l2 x 64 | -delta x 64] floats of the columns
+    static constexpr uint32_t OFF_SC = OFF_BAR + 160;     // DKV: [half][buffer][-l2 x 64 | -delta x 64] floats of the columns
     static constexpr uint32_t BYTES = OFF_SC + ((MODE == 0) ? 0 : 2 * 2 * 2 * 64 * 4);
     static constexpr uint32_t ALLOC = BYTES + 1024;       // slack to align the base to 1 KiB
 };
@@ -104,6 +106,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t bar_acc = bar0 + 120;         // all MMAs done
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_BAR + 128);
     volatile int* abort_word = reinterpret_cast<volatile int*>(smem + L::OFF_BAR + 132);
+    const uint32_t bar_gdone = bar0 + 136;       // [2] DQ: the gradient product that read a dS tile is done
     float* sc_base = reinterpret_cast<float*>(smem + L::OFF_SC);
 
     if (tid == 0) {
@@ -121,6 +124,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_init(bar_efull + 8 * i, MODE == BWD_DQ ? 16 : 8);
         }
         mbar_init(bar_acc, 1);
+        mbar_init(bar_gdone, 1);
+        mbar_init(bar_gdone + 8, 1);
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmQ);
@@ -232,6 +237,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     mbar_wait(bar_cfull + 8 * (t % DQ_KSTAGES), (t / DQ_KSTAGES) & 1, abort_word, p.dev_status);
                     mbar_wait(bar_vfull + 8 * (t % DQ_VSTAGES), (t / DQ_VSTAGES) & 1, abort_word, p.dev_status);
                     if (t > 0) mbar_wait(bar_tfull + 8, (t - 1) & 1, abort_word, p.dev_status);   // S of step t-1 is in registers
+                    // the dP tile of this parity held dS of step t-2 (the two issuing threads have no
+                    // common program order, so its gradient product is waited for)
+                    if (t > 1) mbar_wait(bar_gdone + 8 * (t & 1), ((t - 2) >> 1) & 1, abort_word, p.dev_status);
                     tc_fence_after();
                     if (D == 128) {
                         mma_ss_chain8_fresh(tmem + COL_T1, dr1, smem_desc_sw128(c1, 0, 1024), IDESC_SC128);
@@ -243,19 +251,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     mma_commit(bar_tfull);
                     mma_commit(bar_vempty + 8 * (t % DQ_VSTAGES));      // the V stage is done with
                 };
-                score_full(0);
                 for (int t = 0; t < n_steps; ++t) {
                     if (*abort_word) break;
-                    if (t + 1 < n_steps) score_full(t + 1);
-                    mbar_wait(bar_efull, t & 1, abort_word, p.dev_status);
-                    tc_fence_after();
-                    // A = dS: every thread left its 32 columns' bf16 pairs in the first 16 columns of
-                    // its own 32-column block, so the eight 16-key steps sit at 0, 8, 32, 40, ...
-                    mma_ts_chain8_blocks(tmem + COL_A1, tmem + ((t & 1) ? COL_T2B : COL_T2),
-                                         smem_desc_sw128(stage_k(t), L::ATOM, 1024), IDESC_OUT, t > 0 ? 1u : 0u);
-                    mma_commit(bar_cempty + 8 * (t % DQ_KSTAGES));
+                    score_full(t);
                 }
-                mma_commit(bar_acc);
             } else {
             mbar_wait(bar_cfull, 0, abort_word, p.dev_status);
             tc_fence_after();
@@ -276,6 +275,26 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             mma_commit(bar_acc);
             }
+        }
+        __syncwarp();
+    } else if (warp == 18) {
+        // ------------------------------------------------------------ DQ: gradient-product issuer
+        // A thread of its own, so that its waits and commits do not stand between two score
+        // products in the other issuing thread.
+        if (MODE == BWD_DQ && lane == 0) {
+            for (int t = 0; t < n_steps; ++t) {
+                if (*abort_word) break;
+                mbar_wait(bar_efull, t & 1, abort_word, p.dev_status);
+                tc_fence_after();
+                // A = dS: every thread left its 32 columns' bf16 pairs in the first 16 columns of
+                // its own 32-column block, so the eight 16-key steps sit at 0, 8, 32, 40, ...
+                mma_ts_chain8_blocks(tmem + COL_A1, tmem + ((t & 1) ? COL_T2B : COL_T2),
+                                     smem_desc_sw128(sbase + L::OFF_C + (t % DQ_KSTAGES) * L::TILE, L::ATOM, 1024),
+                                     IDESC_OUT, t > 0 ? 1u : 0u);
+                mma_commit(bar_cempty + 8 * (t % DQ_KSTAGES));
+                mma_commit(bar_gdone + 8 * (t & 1));
+            }
+            mma_commit(bar_acc);
         }
         __syncwarp();
     } else {
