@@ -90,7 +90,7 @@ class ClockSampler(threading.Thread):
     def result(self):
         if not self.ok or not self.sm:
             return {"sm_mhz": None, "sm_max_mhz": self.max_sm, "reasons": ["unavailable"]}
-        return {"sm_mhz": float(np.median(self.sm)), "sm_max_mhz": self.max_sm,
+        return {"sm_mhz": float(np.median(self.sm)), "sm_mhz_min": float(np.min(self.sm)), "sm_max_mhz": self.max_sm,
                 "reasons": sorted(self.reasons), "samples": len(self.sm)}
 
 
