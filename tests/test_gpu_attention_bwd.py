@@ -20,6 +20,8 @@ CASES = {
     "d64_g2": lambda: synth.custom_workload([33, 250], [95, 140], 6, 3, 64, 32, index=51),
     "d128_g1_long": lambda: synth.custom_workload([700], [600], 2, 2, 128, 64, index=52),
     "d128_g16_tiny": lambda: synth.custom_workload([1, 5], [0, 130], 16, 1, 128, 64, index=53),
+    # 21 tiles: the K / V rings of the dQ pass and the stage ring of the dK/dV pass wrap many times
+    "d128_g2_rings": lambda: synth.custom_workload([1300], [1300], 2, 1, 128, 64, index=54),
 }
 
 
