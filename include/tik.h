@@ -48,6 +48,7 @@ typedef int tik_status;
 #define TIK_DEV_BAD_TARGET 2       /* target id outside [0,V): logprob = NaN */
 #define TIK_DEV_WAIT_EXPIRED 4     /* an in-kernel bounded wait ran out (outputs invalid) */
 #define TIK_DEV_BAD_POSITION 8     /* token position outside the cos/sin table: token left untouched */
+#define TIK_DEV_BAD_CONTEXT 16     /* decode: ctx_lens[b] > max_ctx_len: that slot attends keys 0..max_ctx_len-1 only */
 
 #define TIK_OP_ATTN_TRAIN_FWD 0
 #define TIK_OP_ATTN_PREFILL 1
@@ -66,6 +67,11 @@ const char* tik_last_error(const tik_ctx* ctx);
 /* Identifies the numerical contract (tile sizes, MMA shape, exp variant, sum shape).
  * Outputs are bit-comparable only between builds with the same id. */
 const char* tik_contract_id(void);
+
+/* Host-only self-check of the library's per-device launch bookkeeping (no paper counterpart):
+ * kernels that use more than 48 KiB of shared memory are opted in once per (kernel, device), and
+ * this exercises that table with stand-in ordinals.  Needs no GPU.  Returns 0 when it holds. */
+int tik_selftest_host(void);
 
 /* Scratch bytes an operator needs.  rows_or_batch: decode batch B, or log-prob rows T;
  * ignored (0) for train forward / prefill, which need none.  max_ctx: largest context
@@ -164,7 +170,10 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse,
  * 0..ctx_lens[b]-1.  q, o [B][Hq][d]; lse optional fp32 [B][Hq].  A slot with
  * ctx_lens[b] <= 0 is skipped and its output rows are left untouched.  The KV range is
  * split into fixed 2048-key chunks whose partial results go through `ws` and are folded in
- * ascending order by a second kernel on the same stream (fixed-order split-KV combine). */
+ * ascending order by a second kernel on the same stream (fixed-order split-KV combine).
+ * max_ctx_len is a host upper bound on ctx_lens[]: it sizes the grid and the scratch.  A slot
+ * whose ctx_lens[b] exceeds it is computed over keys 0..max_ctx_len-1 only and raises
+ * TIK_DEV_BAD_CONTEXT; nothing is written outside that slot's own scratch and output rows. */
 tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse,
                            const int32_t* ctx_lens, const void* k_cache, const void* v_cache,
                            const int32_t* block_table, int max_blocks, int B, int max_ctx_len,
@@ -223,7 +232,11 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
  *   - All calls on a device share the one scratch array: two calls whose kernels may overlap
  *     on the GPU (different streams) race on it.  Issue them on one stream or order them.
  *   - dev_flags: optional device int that receives TIK_DEV_* flags (OR-ed in; the caller
- *     zeroes and reads it).  NULL sends the flags to a word inside the library.
+ *     zeroes it before the call and reads it afterwards: a word that still holds
+ *     TIK_DEV_WAIT_EXPIRED makes the kernels return at once).  With NULL the flags go to a
+ *     word inside the library that is cleared at the start of every call and that no entry
+ *     point reads: they are DISCARDED, so a bad block-table entry (page read as zeros) or an
+ *     expired wait (outputs invalid) goes unreported.  Pass a word to observe them.
  *   - No error text is kept (there is no context): only the status code is returned. */
 #define TIK_STATIC_SCRATCH_BYTES (8u << 20)
 tik_status tik_attn_decode_static(const void* q, void* o, float* lse, const int32_t* ctx_lens,

@@ -1,4 +1,4 @@
-"""Evaluation-specification harness for the attention kernels (paper Sec. 4.1 and 5.2).
+"""Evaluation-specification harness for the attention kernels (paper Sec. 4.1 and 5.3).
 
 The paper promotes a kernel revision only if it is *verified* (all prescribed correctness checks
 pass), *admissible* (every workload of a fixed set stays within a per-workload slowdown limit of a
@@ -28,9 +28,9 @@ PREFILL_TOKENS = [1024, 4096, 8192, 16384]
 DECODE_CONTEXTS = [128, 1024, 4096, 8192]
 DECODE_BATCHES = [1, 4, 8, 16]
 HEADS = (32, 8, 128, 64)          # Hq, Hkv, head_dim, page size
-MAX_SLOWDOWN = 1.1                # per-workload limit relative to the recorded baseline
-TIMER_STEP_MS = 0.0021            # CUDA-event readings of ~15 us launches move in steps of ~2 us: a workload
-                                  # is over the limit only beyond 1.1x the baseline plus one such step
+MAX_SLOWDOWN = 1.1                # per-workload limit relative to the recorded baseline, no absolute slack
+TRIALS = 5                        # a latency is the mean of five trials (the paper's protocol), each trial
+STATISTIC = "mean of %d trials, each the median of `reps` cold-L2 launches" % TRIALS   # the median of its launches
 
 
 def workload_names() -> List[str]:
@@ -55,9 +55,8 @@ def judge(spec: dict, latencies_ms: Dict[str, float], checks_passed: bool, contr
         preserved = all(recorded.get(k) == v for k, v in hashes.items())
     verified = bool(checks_passed) and preserved is not False
     limit = spec.get("max_slowdown", MAX_SLOWDOWN)
-    step = spec.get("timer_step_ms", TIMER_STEP_MS)
     over = {k: latencies_ms[k] / spec["baseline_ms"][k] for k in spec["baseline_ms"]
-            if k in latencies_ms and latencies_ms[k] > limit * spec["baseline_ms"][k] + step}
+            if k in latencies_ms and latencies_ms[k] > limit * spec["baseline_ms"][k]}
     admissible = verified and not missing and not over
     T = aggregate({k: latencies_ms[k] for k in spec["baseline_ms"] if k in latencies_ms})
     promoted = admissible and T < spec["incumbent_T_ms"]
@@ -73,23 +72,27 @@ def _measure(fn, reps: int = 20, warmup: int = 3, flush=None) -> float:
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
-    times = []
-    for _ in range(reps):
-        if flush is not None:
-            flush.zero_()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        fn()
-        e1.record()
-        torch.cuda.synchronize()
-        times.append(e0.elapsed_time(e1))
-    # the fastest of the repetitions: CUDA-event readings of 15-30 us launches move in ~2 us steps,
-    # and a gate at 1.1x must not trip on that
-    return float(min(times))
+    trials = []
+    for _ in range(TRIALS):
+        times = []
+        for _ in range(reps):
+            if flush is not None:
+                flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        times.sort()
+        trials.append(times[len(times) // 2])
+    # A single CUDA-event reading of a ~15 us launch is coarse (the readings move in ~2 us steps);
+    # the median of a trial's launches and the mean over trials resolve well below the 1.1x gate.
+    return float(sum(trials) / len(trials))
 
 
 def run_grid(reps: int = 20) -> Dict[str, float]:
-    """Latency (ms, cold L2, fastest of `reps`) of every workload of the grid."""
+    """Latency (ms, cold L2; STATISTIC) of every workload of the grid."""
     import numpy as np
     import torch
     from . import binding as tik
@@ -187,7 +190,7 @@ def main() -> None:
     if args.record:
         T = aggregate(lat)
         spec = {"hardware": "B200", "heads": HEADS, "weights": "unit", "max_slowdown": MAX_SLOWDOWN,
-                "baseline_ms": lat, "baseline_T_ms": T, "incumbent_T_ms": T,
+                "statistic": STATISTIC, "reps": args.reps, "baseline_ms": lat, "baseline_T_ms": T, "incumbent_T_ms": T,
                 "hashes": {contract: hashes}, "checks_passed": ok}
         with open(args.record, "w") as f:
             json.dump(spec, f, indent=1)

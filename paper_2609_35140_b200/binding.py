@@ -17,7 +17,7 @@ from . import build as _build
 
 OK = 0
 OP_ATTN_TRAIN_FWD, OP_ATTN_PREFILL, OP_ATTN_DECODE, OP_TOKEN_LOGPROB, OP_ATTN_TRAIN_BWD = 0, 1, 2, 3, 4
-DEV_BAD_BLOCK, DEV_BAD_TARGET, DEV_WAIT_EXPIRED, DEV_BAD_POSITION = 1, 2, 4, 8
+DEV_BAD_BLOCK, DEV_BAD_TARGET, DEV_WAIT_EXPIRED, DEV_BAD_POSITION, DEV_BAD_CONTEXT = 1, 2, 4, 8, 16
 
 _lib = None
 _ctx = {}

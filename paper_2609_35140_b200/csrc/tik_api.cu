@@ -122,6 +122,25 @@ const char* tik_status_str(tik_status s) {
 }
 
 const char* tik_last_error(const tik_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+int tik_selftest_host(void) {
+    // Per-device set-up bookkeeping (DeviceOnce) with stand-in device ordinals and steps: the step
+    // runs once per device, a failed step is retried, a second device is not skipped because the
+    // first one is done, and ordinals outside the table run every time.
+    DeviceOnce once;
+    int runs = 0;
+    auto ok_step = [&]() { ++runs; return cudaSuccess; };
+    auto bad_step = [&]() { ++runs; return cudaErrorInvalidValue; };
+    if (once.run(bad_step, 0) != cudaErrorInvalidValue || runs != 1 || once.is_done(0)) return 1;
+    if (once.run(ok_step, 0) != cudaSuccess || runs != 2 || !once.is_done(0)) return 2;
+    if (once.run(ok_step, 0) != cudaSuccess || runs != 2) return 3;            // done: not run again
+    if (once.is_done(1)) return 4;
+    if (once.run(ok_step, 1) != cudaSuccess || runs != 3 || !once.is_done(1)) return 5;   // second device
+    if (once.run(ok_step, 1) != cudaSuccess || runs != 3) return 6;
+    if (once.run(ok_step, DeviceOnce::MAX_DEVICES + 5) != cudaSuccess || runs != 4) return 7;
+    if (once.run(ok_step, DeviceOnce::MAX_DEVICES + 5) != cudaSuccess || runs != 5) return 8;
+    return 0;
+}
 const char* tik_contract_id(void) { return TIK_CONTRACT_ID; }
 
 size_t tik_workspace_bytes(int op, int64_t rows_or_batch, int Hq, int Hkv, int d, int64_t max_ctx, int H,
@@ -331,6 +350,7 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     p.num_pages = num_pages;
     p.c = scale_to_c(softmax_scale);
     p.nchunk_max = nchunk;
+    p.max_ctx = max_ctx_len;
     p.part_o = static_cast<float*>(ws);
     p.part_ml = p.part_o + static_cast<size_t>(B) * Hq * nchunk * d;
     p.dev_status = ctx->dev_status;

@@ -158,6 +158,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         // a CTA streams `cpc` consecutive chunks; each still leaves its own partial
         chunk = blockIdx.x * p.cpc;
         ctx = p.ctx_lens[seq];
+        if (ctx > p.max_ctx) {
+            // The grid and the scratch were sized from the host's bound: a longer context is cut
+            // to that bound (and flagged) instead of writing partials past the sequence's slots.
+            if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) atomicOr(p.dev_status, TIK_DEV_BAD_CONTEXT);
+            ctx = p.max_ctx;
+        }
         if (ctx <= 0 || chunk * CHUNK >= ctx) return;
         tile_first = chunk * TILES_PER_CHUNK;
         tile_last = min(tile_first + p.cpc * TILES_PER_CHUNK - 1, (ctx - 1) / 128);
@@ -961,7 +967,7 @@ template <int D>
 __global__ void __launch_bounds__(D) combine_kernel(const AttnParams p) {
     pdl_wait();                        // the decode kernel's partials are complete and visible
     const int b = blockIdx.x / p.Hq;
-    const int ctx = p.ctx_lens[b];
+    const int ctx = min(p.ctx_lens[b], p.max_ctx);     // as the decode kernel: never beyond the host's bound
     if (ctx <= 0) return;
     const int nc = (ctx + CHUNK - 1) / CHUNK;
     const long long slot0 = static_cast<long long>(blockIdx.x) * p.nchunk_max;
@@ -1024,14 +1030,14 @@ template <int D, int MODE>
 static cudaError_t launch_attn_t(dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                                  const CUtensorMap& tmV, const AttnParams& p, cudaStream_t stream) {
     auto kern = attn_kernel<D, MODE>;
-    static bool configured = false;   // per instantiation; attribute is per device function
-    cudaError_t e = cudaSuccess;
-    if (!configured) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(AttnSmem<D>::ALLOC));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    // The opt-in to more than 48 KiB of dynamic shared memory belongs to the (function, device)
+    // pair: one flag per device that has launched this instantiation.
+    static DeviceOnce configured;
+    cudaError_t e = configured.run([&]() {
+        return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(AttnSmem<D>::ALLOC));
+    });
+    if (e != cudaSuccess) return e;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;

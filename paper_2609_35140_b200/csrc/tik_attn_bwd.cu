@@ -531,12 +531,13 @@ template <int D, int MODE>
 static cudaError_t launch_bwd_t(dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                                 const CUtensorMap& tmDO, const BwdParams& p, cudaStream_t stream) {
     auto kern = attn_bwd_kernel<D, MODE>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(BwdSmem<D, MODE>::ALLOC));
+    static DeviceOnce configured;     // the opt-in belongs to the (function, device) pair
+    {
+        cudaError_t e = configured.run([&]() {
+            return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(BwdSmem<D, MODE>::ALLOC));
+        });
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     kern<<<grid, BWD_THREADS, BwdSmem<D, MODE>::ALLOC, stream>>>(tmQ, tmK, tmV, tmDO, p);
     return cudaGetLastError();

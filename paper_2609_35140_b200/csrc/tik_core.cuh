@@ -1,7 +1,7 @@
 // The numerical contract shared by every regime (packed train-forward, paged prefill,
 // paged decode, split-KV combine) and by the log-probability kernels.
 //
-// Section 5.2 of the paper lists what decides the bits of unified attention: the
+// Section 5.3 of the paper lists what decides the bits of unified attention: the
 // reduction orders of QK^T, PV, online softmax and final normalisation; where and in
 // which precision scaling and masking happen; the exact exp / reciprocal instructions
 // and flush-to-zero behaviour; the bf16<->fp32 conversion points and the order of

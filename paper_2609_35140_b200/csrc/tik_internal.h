@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <string>
 
 struct tik_ctx {
@@ -16,6 +17,33 @@ struct tik_ctx {
 };
 
 namespace tik {
+
+// Runs a per-device set-up step (typically cudaFuncSetAttribute, whose effect belongs to the
+// current device's context) once for every device that reaches it.  One flag per device ordinal;
+// a failed step is retried by the next call.  Two threads racing on a device's first call may
+// both run the step, which is harmless for idempotent set-up.
+struct DeviceOnce {
+    static constexpr int MAX_DEVICES = 64;
+    std::atomic<bool> done[MAX_DEVICES] = {};
+    bool is_done(int device) const {
+        return device >= 0 && device < MAX_DEVICES && done[device].load(std::memory_order_acquire);
+    }
+    void mark(int device) {
+        if (device >= 0 && device < MAX_DEVICES) done[device].store(true, std::memory_order_release);
+    }
+    // `device` < 0: use the current CUDA device.  Ordinals beyond the table run the step every time.
+    template <class F>
+    cudaError_t run(F&& step, int device = -1) {
+        if (device < 0) {
+            cudaError_t e = cudaGetDevice(&device);
+            if (e != cudaSuccess) return e;
+        }
+        if (is_done(device)) return cudaSuccess;
+        cudaError_t e = step();
+        if (e == cudaSuccess) mark(device);
+        return e;
+    }
+};
 
 // Builds a bf16 tiled tensor map with 128-byte swizzle; dims/box innermost first, strides
 // in bytes for dims 1..rank-1.  Returns false (and fills err) on failure.
@@ -38,6 +66,7 @@ struct AttnParams {
     float* part_ml;              // decode: [B][Hq][nchunk_max][4] = m, l_lo, l_hi, unused
     int page_shift, ppt_shift;   // log2(page_size), log2(pages_per_tile)
     int nchunk_max;
+    int max_ctx;                 // decode: the host's bound on ctx_lens (sized the grid and the scratch)
     int cpc;                     // decode: consecutive chunks streamed by one CTA
     int* dev_status;
     int lookahead;               // train / prefill: block distance of the query-tile L2 prefetch

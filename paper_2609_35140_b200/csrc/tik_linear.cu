@@ -236,12 +236,13 @@ static cudaError_t launch_linear_t(const CUtensorMap& tmA, const CUtensorMap& tm
                                    const LinearParams& p, cudaStream_t stream) {
     using C = lin::Cfg<PAIR>;
     auto kern = linear_kernel<PAIR>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(C::ALLOC));
+    static DeviceOnce configured;     // the opt-in belongs to the (function, device) pair
+    {
+        cudaError_t e = configured.run([&]() {
+            return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(C::ALLOC));
+        });
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     const long long ntile = (p.T + 127) / 128;
     const long long nband = (ntile + lin::BAND - 1) / lin::BAND;

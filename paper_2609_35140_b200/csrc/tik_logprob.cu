@@ -299,12 +299,13 @@ static cudaError_t launch_logprob_main(const CUtensorMap& tmA, const CUtensorMap
                                        cudaStream_t stream) {
     using C = lp::Cfg<PAIR>;
     auto kern = logprob_kernel<PAIR>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(C::ALLOC));
+    static DeviceOnce configured;     // the opt-in belongs to the (function, device) pair
+    {
+        cudaError_t e = configured.run([&]() {
+            return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(C::ALLOC));
+        });
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     const long long ntile = (p.T + 127) / 128;
     const long long nband = (ntile + lp::BAND - 1) / lp::BAND;

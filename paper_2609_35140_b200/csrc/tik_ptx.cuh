@@ -15,6 +15,7 @@ constexpr int TIK_DEV_BAD_BLOCK = 1;      // block-table entry outside [0, num_p
 constexpr int TIK_DEV_BAD_TARGET = 2;     // target id outside [0, V)
 constexpr int TIK_DEV_WAIT_EXPIRED = 4;   // a bounded wait ran out
 constexpr int TIK_DEV_BAD_POSITION = 8;   // token position outside the cos/sin table
+constexpr int TIK_DEV_BAD_CONTEXT = 16;   // decode: ctx_lens[b] above the host's max_ctx_len
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));

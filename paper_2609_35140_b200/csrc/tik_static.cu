@@ -130,6 +130,7 @@ extern "C" tik_status tik_attn_decode_static(const void* q, void* o, float* lse,
     p.num_pages = num_pages;
     p.c = softmax_scale * LOG2E_F;
     p.nchunk_max = nchunk;
+    p.max_ctx = max_ctx_len;
     // Every chunk partial that the combine kernel reads is written by the decode kernel of
     // this same call first, so stale contents of the shared scratch are never consumed.
     p.part_o = static_cast<float*>(s->scratch);

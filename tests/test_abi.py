@@ -39,3 +39,11 @@ def test_host_only_calls_work_without_a_gpu():
     assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 2049) == 16 * 32 * 2 * 132 * 4
     assert binding.workspace_bytes(binding.OP_TOKEN_LOGPROB, 1000, H=4096, V=151936) == 1000 * (2 * 149 + 1) * 4
     assert binding.workspace_bytes(binding.OP_ATTN_TRAIN_FWD, 1000, 8, 2, 128, 4096) == 0
+
+
+def test_per_device_launch_setup_bookkeeping():
+    """The shared-memory opt-in is kept per device: a second GPU of the process is not skipped."""
+    from paper_2609_35140_b200 import binding
+    lib = binding.load()
+    lib.tik_selftest_host.restype = ctypes.c_int
+    assert lib.tik_selftest_host() == 0

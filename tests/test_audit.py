@@ -43,6 +43,16 @@ def test_within_limits_but_not_faster_is_admissible_not_promoted():
     assert tie["admissible"] and not tie["promoted"]            # ties do not replace the incumbent
 
 
+def test_the_gate_has_no_absolute_slack():
+    spec = _spec()
+    lat = dict(spec["baseline_ms"])
+    lat["decode_ctx128_bs1"] = 1.1                      # exactly at the limit: still admissible
+    assert audit.judge(spec, lat, True, "c1", {"a": "h1", "b": "h2"})["admissible"]
+    lat["decode_ctx128_bs1"] = 1.1005                   # 0.5 us over on a 1 ms workload: not admissible
+    v = audit.judge(spec, lat, True, "c1", {"a": "h1", "b": "h2"})
+    assert not v["admissible"] and list(v["over_limit"]) == ["decode_ctx128_bs1"]
+
+
 def test_failed_checks_or_changed_bits_are_not_verified():
     spec = _spec()
     lat = {k: 0.5 for k in spec["baseline_ms"]}

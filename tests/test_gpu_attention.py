@@ -100,8 +100,18 @@ def test_kv_cache_write_is_exact(tik):
     ro = Rollout(tik, w, q, k, v, layout, dirty=3.0)
     upto = [40, 64]
     ro.prefill(stop=upto)
-    kc_ref, vc_ref = synth.fill_paged_cache(w, layout, k, v, upto=upto, fill=3.0)
-    assert torch.equal(bits(ro.kc), bits(kc_ref)) and torch.equal(bits(ro.vc), bits(vc_ref))
+    # expected pool: the oracle's index definition applied to a pool of the same dirty value
+    # (bf16 -> fp32 is exact, so the comparison below is a bit comparison)
+    shape = (layout.num_pages, w.Hkv, layout.page_size, w.d)
+    kc_ref = np.full(shape, 3.0, dtype=np.float32)
+    vc_ref = np.full(shape, 3.0, dtype=np.float32)
+    cu_h = w.cu_seqlens()
+    for s, n in enumerate(upto):
+        sl = slice(int(cu_h[s]), int(cu_h[s]) + n)
+        oracle.paged_scatter(k[sl].float().cpu().numpy(), np.arange(n), layout.block_table[s], layout.page_size, kc_ref)
+        oracle.paged_scatter(v[sl].float().cpu().numpy(), np.arange(n), layout.block_table[s], layout.page_size, vc_ref)
+    assert np.array_equal(ro.kc.float().cpu().numpy(), kc_ref) and np.array_equal(ro.vc.float().cpu().numpy(), vc_ref)
+    assert (kc_ref != 3.0).any() and (kc_ref == 3.0).any()      # rows written and rows left alone both exist
 
 
 def test_invalid_arguments_are_rejected(tik):
@@ -123,3 +133,30 @@ def test_invalid_arguments_are_rejected(tik):
     small = torch.empty(16, dtype=torch.uint8, device="cuda")
     with pytest.raises(tik.TikError):
         tik.tik_attn_decode(q[:2].contiguous(), ctx, kc, vc, bt, 160, w.softmax_scale, ws=small)
+
+
+def test_decode_context_above_the_host_bound_is_cut_and_flagged(tik):
+    """ctx_lens[b] > max_ctx_len: the grid and the scratch were sized from the bound, so that slot
+    is computed over keys 0..max_ctx_len-1 only, TIK_DEV_BAD_CONTEXT is raised, the other slots keep
+    their bits and nothing is written beyond the scratch that the bound asks for."""
+    w = synth.custom_workload([100, 100, 100], [2000, 4500, 1948], 8, 2, 128, 64)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    layout = synth.make_paged_layout(w)
+    bt = torch.from_numpy(layout.block_table).cuda()
+    kc = torch.zeros(layout.num_pages, w.Hkv, layout.page_size, w.d, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    tik.tik_kv_cache_write(k, v, cu, torch.tensor(w.seq_lens, dtype=torch.int32, device="cuda"), kc, vc, bt)
+    cu_h = w.cu_seqlens()
+    bound = 2100                                              # two chunks; sequence 1 holds 4600 keys
+    qd = torch.stack([q[int(cu_h[0]) + 2099], q[int(cu_h[1]) + 2099], q[int(cu_h[2]) + 2047]]).contiguous()
+    good = torch.tensor([2100, 2100, 2048], dtype=torch.int32, device="cuda")
+    ref = tik.tik_attn_decode(qd, good, kc, vc, bt, bound, w.softmax_scale)
+    assert tik.device_status() == 0
+    need = tik.workspace_bytes(tik.OP_ATTN_DECODE, 3, w.Hq, w.Hkv, w.d, bound)
+    ws = torch.full((need + 4096,), 0x5A, dtype=torch.uint8, device="cuda")
+    bad = torch.tensor([2100, 4600, 2048], dtype=torch.int32, device="cuda")     # 3 chunks claimed, 2 allowed
+    out = tik.tik_attn_decode(qd, bad, kc, vc, bt, bound, w.softmax_scale, ws=ws)
+    flags = tik.device_status()
+    assert flags == tik.DEV_BAD_CONTEXT
+    assert count_diff(out, ref) == 0                          # slot 1 cut to the bound, slots 0 and 2 untouched by it
+    assert bool((ws[need:] == 0x5A).all())
