@@ -24,7 +24,10 @@ from . import synth
 
 
 def _time(fn, reps: int, warmup: int, flush):
-    ts = []
+    """Median and minimum launch time in ms.  All repetitions are queued before the one
+    synchronisation, so the host's share of a call (tensor-map encoding, launch) overlaps the
+    previous repetition's L2 flush as it would overlap the previous kernel in a real loop."""
+    evs = []
     for i in range(warmup + reps):
         if flush is not None:
             flush.zero_()
@@ -32,10 +35,9 @@ def _time(fn, reps: int, warmup: int, flush):
         e0.record()
         fn()
         e1.record()
-        torch.cuda.synchronize()
-        if i >= warmup:
-            ts.append(e0.elapsed_time(e1))
-    ts.sort()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    ts = sorted(e0.elapsed_time(e1) for e0, e1 in evs[warmup:])
     return ts[len(ts) // 2], ts[0]
 
 
