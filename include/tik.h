@@ -73,9 +73,11 @@ const char* tik_contract_id(void);
  * this exercises that table with stand-in ordinals.  Needs no GPU.  Returns 0 when it holds. */
 int tik_selftest_host(void);
 
-/* Scratch bytes an operator needs.  rows_or_batch: decode batch B, or log-prob rows T;
- * ignored (0) for train forward / prefill, which need none.  max_ctx: largest context
- * length (decode).  H, V only for the log-prob op.  Returns 0 when no scratch is needed. */
+/* Scratch bytes an operator needs.  rows_or_batch: decode batch B, log-prob rows T, or the number
+ * of sequences S for train forward / prefill.  max_ctx: the host's bound on a context length
+ * (decode, prefill) or sequence length (train forward).  H, V only for the log-prob op.  Returns 0
+ * when no scratch is needed or usable (train forward / prefill outside the range that the
+ * persistent schedule handles: they then run without scratch). */
 size_t tik_workspace_bytes(int op, int64_t rows_or_batch, int Hq, int Hkv, int d,
                            int64_t max_ctx, int H, int V);
 
@@ -88,11 +90,18 @@ tik_status tik_device_status(tik_ctx* ctx, void* stream, int* out_flags);
  *   q [total_tokens][Hq][d], k, v [total_tokens][Hkv][d]  -> o [total_tokens][Hq][d]
  *   lse: optional fp32 [total_tokens][Hq] (natural-log log-sum-exp of the scaled scores)
  *   cu_seqlens: device int32 [S+1]; max_seqlen: host upper bound on any sequence length
- *   (sizes the grid; may be larger than the true maximum). */
+ *   (sizes the grid; may be larger than the true maximum).
+ *   ws, ws_bytes: optional device scratch of tik_workspace_bytes(TIK_OP_ATTN_TRAIN_FWD, S, ...,
+ *   max_seqlen, ...) bytes, 16-byte aligned.  With it the call runs as a persistent kernel (one
+ *   CTA per SM walks a device-built list of work items; the list lives in ws); with NULL, or a
+ *   buffer that is too small, as one CTA per work item.  The output bits are the same: the
+ *   schedule differs, not a row's arithmetic (paper Sec. 5.3: a schedule change must preserve
+ *   bits).  ws is borrowed until the stream-ordered work completes; concurrent calls need
+ *   buffers of their own. */
 tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const void* v, void* o,
                               float* lse, const int32_t* cu_seqlens, int S,
                               int64_t total_tokens, int max_seqlen, int Hq, int Hkv, int d,
-                              float softmax_scale, void* stream);
+                              float softmax_scale, void* ws, size_t ws_bytes, void* stream);
 
 /* Backward of tik_attn_train_fwd (the paper measures the policy-update backward in its layer
  * timings, Sec. 6 Q2, and does not put it under Eq. 1: there is no rollout counterpart).  Given
@@ -157,13 +166,16 @@ tik_status tik_qk_norm_rope_kv_write(tik_ctx* ctx, void* q, void* k, const void*
  * prompt) against the paged cache, which must already hold the keys/values of positions
  * 0 .. ctx_lens[s]-1 (tik_kv_cache_write first).  Query i of sequence s sits at absolute
  * position ctx_lens[s] - q_len[s] + i and attends keys 0..position, so a cached prefix
- * (chunked prefill) is supported.  max_q_len / max_ctx_len: host upper bounds. */
+ * (chunked prefill) is supported.  max_q_len / max_ctx_len: host upper bounds.
+ * ws, ws_bytes: optional scratch as for tik_attn_train_fwd, sized by
+ * tik_workspace_bytes(TIK_OP_ATTN_PREFILL, S, ..., max_ctx_len, ...); same bits with or without. */
 tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse,
                             const int32_t* cu_seqlens_q, const int32_t* ctx_lens,
                             const void* k_cache, const void* v_cache,
                             const int32_t* block_table, int max_blocks, int S, int64_t total_q,
                             int max_q_len, int max_ctx_len, int Hq, int Hkv, int d,
-                            int page_size, int num_pages, float softmax_scale, void* stream);
+                            int page_size, int num_pages, float softmax_scale, void* ws,
+                            size_t ws_bytes, void* stream);
 
 /* Token-wise decode attention (paper Sec. 4.1: the decode entry point): one query token
  * per sequence at position ctx_lens[b]-1 (its own key/value already written) against keys

@@ -51,10 +51,10 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.tik_workspace_bytes.argtypes = [i32, i64, i32, i32, i32, i64, i32, i32]
     lib.tik_workspace_bytes.restype = sz
     lib.tik_device_status.argtypes = [vp, vp, c.POINTER(i32)]
-    lib.tik_attn_train_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, vp]
+    lib.tik_attn_train_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, vp, sz, vp]
     lib.tik_kv_cache_write.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, i32, i32, vp]
     lib.tik_attn_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, i32, i32,
-                                     i32, i32, i32, f32, vp]
+                                     i32, i32, i32, f32, vp, sz, vp]
     lib.tik_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32,
                                     f32, vp, sz, vp]
     lib.tik_qk_norm_rope_kv_write.argtypes = [vp, vp, vp, vp, vp, vp, f32, vp, i32, vp, vp, vp, vp, vp, i32, i32,
@@ -129,19 +129,32 @@ def device_status() -> int:
     return flags.value
 
 
+def _plan_ws(op: int, S: int, max_positions: int, ws, device):
+    """Scratch of the full-sequence kernels: None -> allocate what the op asks for (persistent
+    schedule), False -> pass none (one CTA per work item), a tensor -> use it."""
+    if ws is False:
+        return None
+    if ws is None:
+        need = workspace_bytes(op, S, max_ctx=max_positions)
+        return torch.empty(need, dtype=torch.uint8, device=device) if need > 0 else None
+    return ws
+
+
 def tik_attn_train_fwd(q, k, v, cu_seqlens, max_seqlen: int, softmax_scale: float,
-                       o: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
-    """q [tot,Hq,d], k/v [tot,Hkv,d] bf16, cu_seqlens int32 [S+1] (device) -> o [tot,Hq,d]."""
+                       o: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None, ws=None):
+    """q [tot,Hq,d], k/v [tot,Hkv,d] bf16, cu_seqlens int32 [S+1] (device) -> o [tot,Hq,d].
+    ws: scratch tensor, None (allocated here) or False (run without: one CTA per work item)."""
     ctx = context()
     tot, Hq, d = q.shape
     Hkv = k.shape[1]
     if o is None:
         o = torch.empty_like(q)
     bf = torch.bfloat16
+    ws = _plan_ws(OP_ATTN_TRAIN_FWD, cu_seqlens.numel() - 1, max_seqlen, ws, q.device)
     rc = load().tik_attn_train_fwd(ctx, _ptr(q, bf), _ptr(k, bf), _ptr(v, bf), _ptr(o, bf),
                                    _ptr(lse, torch.float32), _ptr(cu_seqlens, torch.int32),
                                    cu_seqlens.numel() - 1, tot, max_seqlen, Hq, Hkv, d,
-                                   softmax_scale, _stream())
+                                   softmax_scale, _ptr(ws), ws.numel() if ws is not None else 0, _stream())
     _check(rc, ctx)
     return o
 
@@ -238,19 +251,21 @@ def tik_linear(x, weight, y: Optional[torch.Tensor] = None):
 
 def tik_attn_prefill(q, cu_seqlens_q, ctx_lens, k_cache, v_cache, block_table, max_q_len: int,
                      max_ctx_len: int, softmax_scale: float, o: Optional[torch.Tensor] = None,
-                     lse: Optional[torch.Tensor] = None):
-    """q [totq,Hq,d] against the paged cache -> o [totq,Hq,d]."""
+                     lse: Optional[torch.Tensor] = None, ws=None):
+    """q [totq,Hq,d] against the paged cache -> o [totq,Hq,d].  ws as for tik_attn_train_fwd."""
     ctx = context()
     bf = torch.bfloat16
     totq, Hq, d = q.shape
     num_pages, Hkv, page, _ = k_cache.shape
     if o is None:
         o = torch.empty_like(q)
+    ws = _plan_ws(OP_ATTN_PREFILL, ctx_lens.numel(), max_ctx_len, ws, q.device)
     rc = load().tik_attn_prefill(ctx, _ptr(q, bf), _ptr(o, bf), _ptr(lse, torch.float32),
                                  _ptr(cu_seqlens_q, torch.int32), _ptr(ctx_lens, torch.int32),
                                  _ptr(k_cache, bf), _ptr(v_cache, bf), _ptr(block_table, torch.int32),
                                  block_table.shape[1], ctx_lens.numel(), totq, max_q_len, max_ctx_len,
-                                 Hq, Hkv, d, page, num_pages, softmax_scale, _stream())
+                                 Hq, Hkv, d, page, num_pages, softmax_scale, _ptr(ws),
+                                 ws.numel() if ws is not None else 0, _stream())
     _check(rc, ctx)
     return o
 

@@ -59,6 +59,16 @@ static unsigned attn_grid_x(int max_positions) {
     return static_cast<unsigned>(nt <= 16 ? (nt + 1) / 2 : 8 + (nt - 16));
 }
 
+// The persistent kernel runs when the caller passed a large enough, 16-byte aligned plan buffer and
+// the call is within what the planning kernel handles; otherwise one CTA per work item.
+static bool use_persistent(const void* ws, size_t ws_bytes, int S, int max_positions, int Hq) {
+    if (!ws || !aligned16(ws) || !attn_persist_supported(S, max_positions)) return false;
+    const long long nt = (static_cast<long long>(max_positions) + 127) / 128;
+    const long long X = nt <= 16 ? (nt + 1) / 2 : 8 + (nt - 16);
+    if (static_cast<long long>(S) * X * Hq >= (1ll << 31)) return false;
+    return ws_bytes >= attn_plan_bytes(S, max_positions);
+}
+
 static tik_status check_heads(tik_ctx* ctx, int Hq, int Hkv, int d, float scale) {
     if (Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return fail(ctx, TIK_ERR_INVALID_ARG, "Hq must be a positive multiple of Hkv");
     if (!(scale > 0.0f) || !std::isfinite(scale)) return fail(ctx, TIK_ERR_INVALID_ARG, "softmax_scale must be finite and > 0");
@@ -147,6 +157,11 @@ size_t tik_workspace_bytes(int op, int64_t rows_or_batch, int Hq, int Hkv, int d
                            int V) {
     (void)Hkv;
     (void)H;
+    if (op == TIK_OP_ATTN_TRAIN_FWD || op == TIK_OP_ATTN_PREFILL) {
+        // rows_or_batch = number of sequences S, max_ctx = the host's bound on a sequence's positions
+        if (rows_or_batch <= 0 || max_ctx <= 0 || !attn_persist_supported(rows_or_batch, max_ctx)) return 0;
+        return attn_plan_bytes(rows_or_batch, max_ctx);
+    }
     if (op == TIK_OP_ATTN_DECODE) {
         if (rows_or_batch <= 0 || max_ctx <= 0) return 0;
         const int64_t nchunk = (max_ctx + CHUNK - 1) / CHUNK;
@@ -178,7 +193,7 @@ tik_status tik_device_status(tik_ctx* ctx, void* stream, int* out_flags) {
 
 tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const void* v, void* o, float* lse,
                               const int32_t* cu_seqlens, int S, int64_t total_tokens, int max_seqlen, int Hq,
-                              int Hkv, int d, float softmax_scale, void* stream) {
+                              int Hkv, int d, float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
     if (!ctx) return TIK_ERR_INVALID_ARG;
     if (S < 0 || total_tokens < 0 || max_seqlen < 0) return fail(ctx, TIK_ERR_INVALID_ARG, "negative size");
     tik_status s = check_heads(ctx, Hq, Hkv, d, softmax_scale);
@@ -213,7 +228,12 @@ tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const 
     p.lookahead = ctx->sm_count;
     dim3 grid(attn_grid_x(max_seqlen), Hq, S);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
-    cudaError_t e = launch_attn(d, 0, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
+    cudaError_t e;
+    if (use_persistent(ws, ws_bytes, S, max_seqlen, Hq))
+        e = launch_attn_persist(d, false, ctx->sm_count, S, static_cast<int>(grid.x), tmQ, tmK, tmV, p, ws,
+                                static_cast<cudaStream_t>(stream));
+    else
+        e = launch_attn(d, 0, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_train_fwd");
 }
 
@@ -255,7 +275,7 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
                             const int32_t* ctx_lens, const void* k_cache, const void* v_cache,
                             const int32_t* block_table, int max_blocks, int S, int64_t total_q, int max_q_len,
                             int max_ctx_len, int Hq, int Hkv, int d, int page_size, int num_pages,
-                            float softmax_scale, void* stream) {
+                            float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
     if (!ctx) return TIK_ERR_INVALID_ARG;
     if (S < 0 || total_q < 0 || max_q_len < 0 || max_ctx_len < 0 || max_blocks < 0 || num_pages < 0)
         return fail(ctx, TIK_ERR_INVALID_ARG, "negative size");
@@ -301,7 +321,12 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
     // query tiles are aligned to absolute positions 0 .. ctx-1 (tiles before the first new token exit)
     dim3 grid(attn_grid_x(max_ctx_len), Hq, S);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
-    cudaError_t e = launch_attn(d, 1, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
+    cudaError_t e;
+    if (use_persistent(ws, ws_bytes, S, max_ctx_len, Hq))
+        e = launch_attn_persist(d, true, ctx->sm_count, S, static_cast<int>(grid.x), tmQ, tmK, tmV, p, ws,
+                                static_cast<cudaStream_t>(stream));
+    else
+        e = launch_attn(d, 1, grid, tmQ, tmK, tmV, p, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_prefill");
 }
 

@@ -77,6 +77,16 @@ cudaError_t launch_attn(int d, int mode, dim3 grid, const CUtensorMap& tmQ, cons
                         const CUtensorMap& tmV, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_combine(int d, const AttnParams& p, int B, cudaStream_t stream);
 
+// Persistent full-sequence attention (tik_attn_persist.cu): a planning kernel writes the list of
+// work items of the call into `plan` (attn_plan_bytes bytes, 16-byte aligned), then one CTA per SM
+// walks it.  X = candidate items per sequence for the host's length bound (as the grid's x extent
+// of the one-CTA-per-item kernel).  Same output bits as launch_attn.
+size_t attn_plan_bytes(int64_t S, int64_t max_positions);
+bool attn_persist_supported(int64_t S, int64_t max_positions);
+cudaError_t launch_attn_persist(int d, bool paged, int sm_count, int S, int X, const CUtensorMap& tmQ,
+                                const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnParams& p, void* plan,
+                                cudaStream_t stream);
+
 struct PrepParams {
     __nv_bfloat16* q;            // [total_new][Hq][d], in place
     __nv_bfloat16* k;            // [total_new][Hkv][d], in place
