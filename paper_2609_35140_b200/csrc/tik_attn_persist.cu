@@ -44,7 +44,7 @@ struct PASmem {
 // Event trace of one CTA (debug builds only, -DTIK_PA_TRACE): clock64 stamps of the roles' key
 // events for the CTA's first items, read back through tik_debug_pa_trace.
 #ifdef TIK_PA_TRACE
-constexpr int PA_TRACE_ITEMS = 48, PA_TRACE_EVENTS = 32;
+constexpr int PA_TRACE_ITEMS = 48, PA_TRACE_EVENTS = 48;
 __device__ long long g_pa_trace[PA_TRACE_ITEMS * PA_TRACE_EVENTS];
 #define PA_STAMP(k, ev)                                                                         \
     do {                                                                                        \
@@ -236,7 +236,7 @@ __device__ __noinline__ void pa_fold_o_tmem(uint32_t t_a, uint32_t t_b, FoldCoef
 template <int NCOLS>
 __device__ __noinline__ void pa_store_rows(uint32_t acc, float inv, int row0, int lo, int hi, int head, int col0, int D,
                                            uint8_t* stage, __nv_bfloat16* o, int Hq, uint32_t odrain_bar,
-                                           uint32_t odrain_n, int lane, int quarter) {
+                                           uint32_t odrain_n, int lane, int quarter, long long* tr = nullptr) {
     constexpr int PASS = NCOLS < 64 ? NCOLS : 64;      // columns per pass
     constexpr int NCH = PASS / 8;                       // 16-byte chunks per row and pass
     constexpr int RPI = 32 / NCH;                       // rows per store instruction
@@ -247,6 +247,7 @@ __device__ __noinline__ void pa_store_rows(uint32_t acc, float inv, int row0, in
         for (int cc = 0; cc < PASS / 32; ++cc)
             tmem_ld32(acc + PASS * a + 32 * cc, *reinterpret_cast<uint32_t(*)[32]>(&v[32 * cc]));
         tmem_wait_ld();
+        if (tr) tr[3 * a] = clock64();
         if (a == NCOLS / PASS - 1) {
             tc_fence_before();
             __syncwarp();
@@ -263,16 +264,25 @@ __device__ __noinline__ void pa_store_rows(uint32_t acc, float inv, int row0, in
                 make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
         __syncwarp();
+        if (tr) tr[3 * a + 1] = clock64();
         const int cl = lane % NCH, r0 = lane / NCH;
+        uint4 val[NCH];
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
             const int row = r0 + RPI * i;               // row of this warp's 32
-            const int trow = 32 * quarter + row;        // row of the tile
-            const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (NCH * 16) + ((cl ^ (row & (NCH - 1))) << 4));
-            if (trow >= lo && trow < hi)
-                *reinterpret_cast<uint4*>(o + (static_cast<long long>(row0 + trow) * Hq + head) * D + col0 + PASS * a + cl * 8) = val;
+            val[i] = *reinterpret_cast<const uint4*>(stage + row * (NCH * 16) + ((cl ^ (row & (NCH - 1))) << 4));
+        }
+        // all rows are read back before the first store is issued (the compiler cannot move a shared
+        // load across a global store on its own)
+        __nv_bfloat16* const gp = o + (static_cast<long long>(row0 + 32 * quarter + r0) * Hq + head) * D + col0 + PASS * a + cl * 8;
+        const long long pitch = static_cast<long long>(RPI) * Hq * D;
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const int trow = 32 * quarter + r0 + RPI * i;        // row of the tile
+            if (trow >= lo && trow < hi) *reinterpret_cast<uint4*>(gp + i * pitch) = val[i];
         }
         __syncwarp();
+        if (tr) tr[3 * a + 2] = clock64();
     }
 }
 
@@ -693,8 +703,14 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     const int e_row0 = m[0], e_lo = m[1], e_hi = m[2], e_head = m[3];
                     if (r >= e_lo && r < e_hi && p.lse)
                         p.lse[(static_cast<long long>(e_row0) + r) * p.Hq + e_head] = finalize_lse(m_run, Ltot, c);
+#ifdef TIK_PA_TRACE
+                    long long* tr = (blockIdx.x == 0 && k < PA_TRACE_ITEMS && quarter == 0 && lane == 0)
+                                        ? &g_pa_trace[k * PA_TRACE_EVENTS + 32 + 8 * wg] : nullptr;
+#else
+                    long long* tr = nullptr;
+#endif
                     pa_store_rows<D>(to, inv, e_row0, e_lo, e_hi, e_head, 0, D, stage_warp, o_base, p.Hq,
-                                     bar_odrain + 8 * wg, 2u, lane, quarter);
+                                     bar_odrain + 8 * wg, 2u, lane, quarter, tr);
                 }
                 if (quarter == 0 && lane == 0) PA_STAMP(k, 17 + 10 * wg);
             } else {

@@ -22,6 +22,9 @@ CASES = {
     "d128_g16_tiny": lambda: synth.custom_workload([1, 5], [0, 130], 16, 1, 128, 64, index=53),
     # 21 tiles: the K / V rings of the dQ pass and the stage ring of the dK/dV pass wrap many times
     "d128_g2_rings": lambda: synth.custom_workload([1300], [1300], 2, 1, 128, 64, index=54),
+    # head_dim 64 over 18 tiles, and a grouped-query sequence longer than one 2048-key chunk
+    "d64_g2_18tiles": lambda: synth.custom_workload([1100], [1150], 4, 2, 64, 32, index=55),
+    "d128_g4_multichunk": lambda: synth.custom_workload([900, 40], [1700, 9], 4, 1, 128, 64, index=56),
 }
 
 

@@ -23,7 +23,7 @@ def tik():
 def _oracle_rows(w, q, k, v, rows):
     """Oracle outputs for (sequence, head, position) rows, copying only the K/V slices they need."""
     cu = w.cu_seqlens()
-    ks, vs, qs, off, ln = [], [], [], [], []
+    ks, vs, off, ln = [], [], [], []
     base = 0
     cache = {}
     for (s, h, t) in rows:
@@ -34,10 +34,12 @@ def _oracle_rows(w, q, k, v, rows):
             vs.append(v[sl, g].float().cpu().numpy())
             cache[(s, g)] = base
             base += w.seq_lens[s]
-        qs.append(q[int(cu[s]) + t, h].float().cpu().numpy())
         off.append(cache[(s, g)])
         ln.append(t + 1)
-    out, _ = oracle.attn_rows(np.stack(qs), np.concatenate(ks), np.concatenate(vs), off, ln, w.softmax_scale)
+    idx = torch.tensor([int(cu[s]) + t for (s, h, t) in rows], device=q.device)
+    hd = torch.tensor([h for (s, h, t) in rows], device=q.device)
+    qs = q[idx, hd].float().cpu().numpy()
+    out, _ = oracle.attn_rows(qs, np.concatenate(ks), np.concatenate(vs), off, ln, w.softmax_scale)
     return out
 
 
@@ -48,22 +50,31 @@ def test_attention_at_full_size(tik, index):
     cu_h = w.cu_seqlens()
     o_train = tik.tik_attn_train_fwd(q, k, v, cu, max(w.seq_lens), w.softmax_scale)
 
-    # --- oracle on sampled rows (boundaries of tiles, pages and chunks, first/last rows, random)
+    # --- oracle: every position of the two shortest and the longest sequence for one query head per
+    # KV head, plus >= 4096 seeded (sequence, head, position) rows that include every sequence's first
+    # and last row and the rows around tile (128), page and chunk (2048) boundaries
     rng = np.random.default_rng(w.seed + 17)
-    seqs = sorted(set([int(np.argmin(w.seq_lens)), int(np.argmax(w.seq_lens))] +
-                      [int(x) for x in rng.integers(0, w.S, 2)]))
+    order = np.argsort(w.seq_lens, kind="stable")
+    whole = sorted({int(order[0]), int(order[1]), int(order[-1])})
     rows = []
-    for s in seqs:
-        L = w.seq_lens[s]
-        marks = [0, 1, 63, 64, 127, 128, 129, w.prompt_lens[s] - 1, w.prompt_lens[s], 2047, 2048, 2049,
-                 4095, 4096, L // 2, L - 2, L - 1] + [int(x) for x in rng.integers(0, L, 6)]
-        for t in marks:
-            if 0 <= t < L:
-                rows.append((s, int(rng.integers(0, w.Hq)), t))
-    ref = _oracle_rows(w, q, k, v, rows)
-    got = torch.stack([o_train[int(cu_h[s]) + t, h] for (s, h, t) in rows]).float().cpu().numpy()
-    assert np.abs(got - ref).max() <= ATTN_TOL
-    del ref, got
+    for s in whole:
+        heads = [g * w.G + int(rng.integers(0, w.G)) for g in range(w.Hkv)]
+        rows += [(s, h, t) for h in heads for t in range(w.seq_lens[s])]
+    n_whole = len(rows)
+    rows += synth.sample_rows(w, 4096)
+    assert len(rows) - n_whole >= 4096
+    seqs = whole
+    step = 40000                      # bounded host copies: the oracle takes the rows in slices
+    worst = 0.0
+    for a in range(0, len(rows), step):
+        part = rows[a:a + step]
+        ref = _oracle_rows(w, q, k, v, part)
+        idx = torch.tensor([int(cu_h[s]) + t for (s, h, t) in part], device="cuda")
+        hd = torch.tensor([h for (s, h, t) in part], device="cuda")
+        got = o_train[idx, hd].float().cpu().numpy()
+        worst = max(worst, float(np.abs(got - ref).max()))
+        del ref, got
+    assert worst <= ATTN_TOL, worst
 
     # --- rollout: cache write, prefill of one prompt per group, decode at sampled positions
     layout = synth.make_paged_layout(w)
@@ -112,8 +123,8 @@ def test_logprob_at_full_size(tik, index):
     T = hidden.shape[0]
     lp = tik.tik_token_logprob(hidden, W, target)
     rng = np.random.default_rng(w.seed + 23)
-    n = 48 if index <= 2 else 24
-    sample = np.unique(np.concatenate([[0, 127, 128, T - 1], rng.integers(0, T, n)]))
+    sample = np.unique(np.concatenate([[0, 127, 128, T - 1], rng.integers(0, T, 520)]))
+    assert len(sample) >= 512
     st = torch.from_numpy(sample).cuda()
     ref, _ = oracle.token_logprob(hidden[st].float().cpu().numpy(), W.float().cpu().numpy(),
                                   target[st].cpu().numpy())
@@ -123,6 +134,24 @@ def test_logprob_at_full_size(tik, index):
     for a, b in [(0, 1), (0, w.S), (T - 300, T), (1000, 1000 + 64)]:
         part = tik.tik_token_logprob(hidden[a:b].contiguous(), W, target[a:b].contiguous())
         assert count_diff(part, lp[a:b]) == 0, (a, b)
+
+
+@pytest.mark.parametrize("index,group", [(1, None), (2, 3)])
+def test_step_by_step_rollout_at_full_size(tik, index, group):
+    """Eq. 1 at full size: prefill the prompts, then decode EVERY response token step by step (cache
+    write + decode + combine per step, the batch shrinking as sequences finish); every row of the
+    replay must equal the packed train-forward's row bit for bit.  configs[1] whole; of configs[2] one
+    GRPO group (8 responses behind one shared prompt), with the heads and page size of the workload."""
+    from gpu_common import Rollout
+    w = synth.get_workload(index)
+    if group is not None:
+        ids = [s for s, g in enumerate(w.group_of) if g == group]
+        w = synth.custom_workload([w.prompt_lens[s] for s in ids], [w.response_lens[s] for s in ids], w.Hq, w.Hkv,
+                                  w.d, w.page_size, group_of=[0] * len(ids), index=200 + index)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    o_train = tik.tik_attn_train_fwd(q, k, v, cu, max(w.seq_lens), w.softmax_scale)
+    o_roll = Rollout(tik, w, q, k, v, synth.make_paged_layout(w)).replay()
+    assert count_diff(o_train, o_roll) == 0
 
 
 def test_attention_backward_at_full_size(tik):
@@ -145,3 +174,30 @@ def test_attention_backward_at_full_size(tik):
             err = got.float().cpu().numpy().astype(np.float64) - ref
             assert np.abs(err).max() <= 2e-2 * np.abs(ref).max()
             assert np.sqrt((err ** 2).mean()) <= 6e-3 * np.sqrt((ref ** 2).mean())
+
+
+@pytest.mark.parametrize("index", [2, 3])
+def test_attention_backward_on_larger_workloads(tik, index):
+    """Workloads 2 and 3 at their real sizes.  Workload 2: the oracle checks its shortest sequence whole
+    (all heads; sequences are independent).  Workload 3's sequences have 16 384 tokens, beyond what the
+    fp64 oracle can take whole: it checks dQ of the first 2 600 positions (two chunks) of one sequence,
+    which depend on that prefix only (row i of dQ involves keys 0..i), through the oracle on the prefix."""
+    w = synth.get_workload(index)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    do, _, _, _ = synth.make_qkv(w, "cuda", seed_offset=5)
+    lse = torch.empty(q.shape[0], w.Hq, dtype=torch.float32, device="cuda")
+    o = tik.tik_attn_train_fwd(q, k, v, cu, max(w.seq_lens), w.softmax_scale, lse=lse)
+    dq, dk, dv = tik.tik_attn_train_bwd(q, k, v, o, do, lse, cu, max(w.seq_lens), w.softmax_scale)
+    assert bool(torch.isfinite(dq).all() and torch.isfinite(dk).all() and torch.isfinite(dv).all())
+    cu_h = w.cu_seqlens()
+    s = int(np.argmin(w.seq_lens))
+    n = w.seq_lens[s] if index == 2 else 2600
+    sl = slice(int(cu_h[s]), int(cu_h[s]) + n)
+    rq, rk, rv = oracle.attn_bwd_packed(q[sl].float().cpu().numpy(), k[sl].float().cpu().numpy(),
+                                        v[sl].float().cpu().numpy(), do[sl].float().cpu().numpy(),
+                                        np.array([0, n], dtype=np.int32), w.softmax_scale)
+    pairs = ((dq[sl], rq),) if index == 3 else ((dq[sl], rq), (dk[sl], rk), (dv[sl], rv))
+    for got, ref in pairs:
+        err = got.float().cpu().numpy().astype(np.float64) - ref
+        assert np.abs(err).max() <= 2e-2 * np.abs(ref).max()
+        assert np.sqrt((err ** 2).mean()) <= 6e-3 * np.sqrt((ref ** 2).mean())
