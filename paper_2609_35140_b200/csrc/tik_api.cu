@@ -169,8 +169,11 @@ size_t tik_workspace_bytes(int op, int64_t rows_or_batch, int Hq, int Hkv, int d
     }
     if (op == TIK_OP_TOKEN_LOGPROB) {
         if (rows_or_batch <= 0 || V <= 0) return 0;
-        const int64_t nsuper = (V + LP_SUPER - 1) / LP_SUPER;
-        return static_cast<size_t>(rows_or_batch) * (2 * nsuper + 1) * sizeof(float);
+        // partial (max, sum) pairs: per 1024-column super-chunk, or per 128-column tile for calls of
+        // at most LP_UNIT_MODE_ROWS rows (decode-sized batches), plus one target logit per row
+        const int64_t nsuper = (V + LP_SUPER - 1) / LP_SUPER, ntile = (V + LP_TILE - 1) / LP_TILE;
+        const int64_t npart = rows_or_batch <= LP_UNIT_MODE_ROWS ? ntile : nsuper;
+        return static_cast<size_t>(rows_or_batch) * (2 * npart + 1) * sizeof(float);
     }
     if (op == TIK_OP_ATTN_TRAIN_BWD) {      // rows_or_batch = total tokens: delta [tokens][Hq]
         if (rows_or_batch <= 0) return 0;
@@ -483,8 +486,12 @@ tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_he
         const long long ntile = (T + 127) / 128;
         while (p.spc < 8 && ntile * ((p.nsuper + 2 * p.spc - 1) / (2 * p.spc)) >= 4ll * ctx->sm_count) p.spc *= 2;
     }
+    p.unit_mode = T <= LP_UNIT_MODE_ROWS ? 1 : 0;
+    p.nunit = (V + 255) / 256;
+    p.ntile128 = (V + LP_TILE - 1) / LP_TILE;
+    p.sm_count = ctx->sm_count;
     p.part_ml = static_cast<float*>(ws);
-    p.z_target = p.part_ml + static_cast<size_t>(T) * p.nsuper * 2;
+    p.z_target = p.part_ml + static_cast<size_t>(T) * (p.unit_mode ? p.ntile128 : p.nsuper) * 2;
     p.inv_temperature = inv_temperature;
     p.dev_status = ctx->dev_status;
     cudaError_t e = launch_logprob(tmA, tmB, p, pair, static_cast<cudaStream_t>(stream));

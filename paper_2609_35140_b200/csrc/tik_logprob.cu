@@ -64,8 +64,18 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int tile_in_band = static_cast<int>(rem % BAND);
     // (a pair leaves only together: a lone tile at the end of T keeps its partner, whose rows lie
     // past T, arrive as zeros and are never stored)
-    if ((PAIR ? (tile_in_band & ~1) : tile_in_band) >= band_tiles) return;
-    const int tok0 = (band * BAND + tile_in_band) * 128;
+    // Unit mode (calls of one or two token tiles, i.e. decode-sized batches): such a call streams all
+    // of lm_head once and is bound by HBM, and V / 1024 super-chunks do not divide over the SMs (149
+    // on 148: a second wave for one CTA).  There a CTA (pair) is persistent and takes the 256-column
+    // accumulator steps u, u + n, u + 2n, ... of the vocabulary; every 128-column tile leaves its own
+    // (max, sum) pair and the finish kernel folds them in the fixed order (tiles ascending inside a
+    // super-chunk, then super-chunks ascending): the same operations on the same numbers.
+    const bool unit_mode = p.unit_mode != 0;
+    const int u_first = static_cast<int>(blockIdx.x) / (PAIR ? 2 : 1);
+    const int u_stride = static_cast<int>(gridDim.x) / (PAIR ? 2 : 1);
+    const int n_my_units = unit_mode ? (u_first < p.nunit ? (p.nunit - 1 - u_first) / u_stride + 1 : 0) : 0;
+    if (!unit_mode && (PAIR ? (tile_in_band & ~1) : tile_in_band) >= band_tiles) return;
+    const int tok0 = unit_mode ? (PAIR ? 128 * static_cast<int>(rank) : 0) : (band * BAND + tile_in_band) * 128;
     // 256-column accumulator steps of super-chunk sup0 + sp
     auto n_nt_of = [&](int sp) { return min(LP_SUPER / NB, (p.V - (sup0 + sp) * LP_SUPER + NB - 1) / NB); };
     const int n_kb = p.H / 64;
@@ -120,9 +130,11 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int sp = 0; sp < n_sp; ++sp)
-            for (int nt = 0; nt < n_nt_of(sp); ++nt) {
-                const int col0 = (sup0 + sp) * LP_SUPER + nt * NB;
+            // accumulator steps of this CTA: unit mode a strided list, else spc super-chunks x up to 4
+            const int n_sp_loop = unit_mode ? n_my_units : n_sp;
+            for (int sp = 0; sp < n_sp_loop; ++sp)
+            for (int nt = 0; nt < (unit_mode ? 1 : n_nt_of(sp)); ++nt) {
+                const int col0 = unit_mode ? (u_first + sp * u_stride) * NB : (sup0 + sp) * LP_SUPER + nt * NB;
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
                     const int s = it % STAGES;
@@ -147,8 +159,9 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, acc = 0;              // acc counts accumulator steps across super-chunks
-            for (int sp = 0; sp < n_sp; ++sp)
-            for (int nt = 0; nt < n_nt_of(sp); ++nt, ++acc) {
+            const int n_sp_loop = unit_mode ? n_my_units : n_sp;
+            for (int sp = 0; sp < n_sp_loop; ++sp)
+            for (int nt = 0; nt < (unit_mode ? 1 : n_nt_of(sp)); ++nt, ++acc) {
                 const int buf = acc & 1;
                 const uint32_t use = acc >> 1;
                 if (use > 0) mbar_wait(bar_acc_empty + 8 * buf, (use - 1) & 1, abort_word, p.dev_status);
@@ -187,11 +200,12 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int target = row_valid ? p.target[t] : -1;
         const float it_scale = p.inv_temperature;
         uint32_t acc = 0;
-        for (int sp = 0; sp < n_sp; ++sp) {
-        const int col_base = (sup0 + sp) * LP_SUPER;
+        const int n_sp_loop = unit_mode ? n_my_units : n_sp;
+        for (int sp = 0; sp < n_sp_loop; ++sp) {
+        const int col_base = unit_mode ? (u_first + sp * u_stride) * NB : (sup0 + sp) * LP_SUPER;
         float M = -CUDART_INF_F, Lsum = 0.0f;
         bool first = true;
-        for (int nt = 0; nt < n_nt_of(sp); ++nt, ++acc) {
+        for (int nt = 0; nt < (unit_mode ? 1 : n_nt_of(sp)); ++nt, ++acc) {
             const int buf = acc & 1;
             mbar_wait(bar_acc_full + 8 * buf, (acc >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
@@ -234,7 +248,14 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
                 const float lt = rs.total();
-                if (first) {
+                if (unit_mode) {
+                    // the tile's own pair; folded later by the finish kernel
+                    if (row_valid) {
+                        const long long slot = t * p.ntile128 + (col0 >> 7);
+                        p.part_ml[2 * slot] = mt;
+                        p.part_ml[2 * slot + 1] = lt;
+                    }
+                } else if (first) {
                     M = mt;
                     Lsum = lt;
                     first = false;
@@ -250,7 +271,7 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (PAIR) mbar_arrive_cluster(lead_acc_empty + 8 * buf);
             else mbar_arrive(bar_acc_empty + 8 * buf);
         }
-        if (row_valid) {
+        if (row_valid && !unit_mode) {
             p.part_ml[2 * (t * p.nsuper + sup0 + sp)] = M;
             p.part_ml[2 * (t * p.nsuper + sup0 + sp) + 1] = Lsum;
         }
@@ -294,6 +315,66 @@ __global__ void __launch_bounds__(256) logprob_finish_kernel(const LogprobParams
     }
 }
 
+// Unit mode: one block per token.  Thread s folds the tiles of super-chunk s in ascending order
+// (first tile copied, the others folded: the main kernel's in-CTA sequence), then thread 0 folds
+// the super-chunks in ascending order as logprob_finish_kernel does.
+__global__ void __launch_bounds__(256) logprob_finish_tiles_kernel(const LogprobParams p) {
+    pdl_wait();
+    __shared__ float sm[256], sl[256];
+    const long long t = blockIdx.x;
+    const float* ml = p.part_ml + 2 * t * p.ntile128;
+    constexpr int TPS = LP_SUPER / LP_TILE;        // tiles per super-chunk
+    for (int s0 = 0; s0 < p.nsuper; s0 += 256) {
+        const int s = s0 + threadIdx.x;
+        float M = 0.0f, Lsum = 0.0f;
+        if (s < p.nsuper) {
+            const int t0 = s * TPS, t1 = min(p.ntile128, t0 + TPS);
+            M = ml[2 * t0];
+            Lsum = ml[2 * t0 + 1];
+            for (int j = t0 + 1; j < t1; ++j) {
+                const FoldCoef f = fold_coef(M, ml[2 * j], LOG2E_F);
+                Lsum = fold_value(Lsum, ml[2 * j + 1], f);
+                M = f.M_new;
+            }
+        }
+        __syncthreads();                            // (the previous batch of super-chunks has been consumed)
+        sm[threadIdx.x] = M;
+        sl[threadIdx.x] = Lsum;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            // running total kept in sm[0] / sl[0] across batches of 256 super-chunks
+            float Mt = sm[0], Lt = sl[0];
+            if (s0 > 0) {
+                // restore the running total saved below, then fold this batch's first entry
+                const float Mr = p.part_ml[2 * t * p.ntile128], Lr = p.part_ml[2 * t * p.ntile128 + 1];
+                const FoldCoef f = fold_coef(Mr, Mt, LOG2E_F);
+                Lt = fold_value(Lr, Lt, f);
+                Mt = f.M_new;
+            }
+            const int n = min(256, p.nsuper - s0);
+            for (int i = 1; i < n; ++i) {
+                const FoldCoef f = fold_coef(Mt, sm[i], LOG2E_F);
+                Lt = fold_value(Lt, sl[i], f);
+                Mt = f.M_new;
+            }
+            if (s0 + 256 < p.nsuper) {              // more batches follow: park the running total
+                p.part_ml[2 * t * p.ntile128] = Mt;
+                p.part_ml[2 * t * p.ntile128 + 1] = Lt;
+            } else {
+                const float lse = lp_lse(Mt, Lt);
+                if (p.lse) p.lse[t] = lse;
+                const int target = p.target[t];
+                if (target < 0 || target >= p.V) {
+                    atomicOr(p.dev_status, TIK_DEV_BAD_TARGET);
+                    p.logprob[t] = CUDART_NAN_F;
+                } else {
+                    p.logprob[t] = __fsub_rn(p.z_target[t], lse);
+                }
+            }
+        }
+    }
+}
+
 template <bool PAIR>
 static cudaError_t launch_logprob_main(const CUtensorMap& tmA, const CUtensorMap& tmB, const LogprobParams& p,
                                        cudaStream_t stream) {
@@ -309,7 +390,11 @@ static cudaError_t launch_logprob_main(const CUtensorMap& tmA, const CUtensorMap
     }
     const long long ntile = (p.T + 127) / 128;
     const long long nband = (ntile + lp::BAND - 1) / lp::BAND;
-    const long long grid = nband * lp::BAND * ((p.nsuper + p.spc - 1) / p.spc);   // even: BAND is
+    long long grid = nband * lp::BAND * ((p.nsuper + p.spc - 1) / p.spc);   // even: BAND is
+    if (p.unit_mode) {       // persistent CTAs (pairs), one per SM (two SMs), never more than there are units
+        const long long slots = PAIR ? p.sm_count / 2 : p.sm_count;
+        grid = (slots < p.nunit ? slots : p.nunit) * (PAIR ? 2 : 1);
+    }
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = PAIR ? 2 : 1;
@@ -335,11 +420,12 @@ cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(static_cast<unsigned>((p.T + 255) / 256));
+    cfg.gridDim = dim3(static_cast<unsigned>(p.unit_mode ? p.T : (p.T + 255) / 256));
     cfg.blockDim = dim3(256);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (p.unit_mode) return cudaLaunchKernelEx(&cfg, logprob_finish_tiles_kernel, p);
     return cudaLaunchKernelEx(&cfg, logprob_finish_kernel, p);
 }
 

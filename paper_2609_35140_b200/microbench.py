@@ -1,7 +1,7 @@
 """Single-kernel timings of the library on chosen shapes (also the command line for profiler captures).
 
 Each case builds seeded synthetic inputs on the GPU, runs one entry point `--warmup` + `--reps`
-times with a 512 MiB buffer overwritten before every launch (L2 flush, outside the timed span),
+times with an L2 flush before every launch (512 MiB written, then 256 MiB read; outside the timed span),
 times every launch with CUDA events on the launching stream and prints one JSON line with the
 median and minimum, the algorithmic work and the resulting rate.
 
@@ -21,6 +21,22 @@ import torch
 
 from . import binding as tik
 from . import synth
+
+
+class L2Flush:
+    """Cold, clean L2 before a timed launch: a 512 MiB buffer is overwritten (nothing of the timed
+    kernel's inputs survives in the 126 MB L2), then a 256 MiB buffer is read, which pushes the
+    first pass's dirty lines out to HBM.  Without the read pass the timed kernel pays for writing
+    back up to an L2-ful of the flush's own data (~15 us of HBM time on a B200)."""
+
+    def __init__(self, device="cuda", read_pass: bool = True):
+        self.w = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+        self.r = torch.zeros(64 << 20, dtype=torch.int32, device=device) if read_pass else None
+
+    def zero_(self):            # same call as the plain buffer it replaces
+        self.w.zero_()
+        if self.r is not None:
+            torch.sum(self.r)
 
 
 def _time(fn, reps: int, warmup: int, flush):
@@ -66,7 +82,7 @@ def paged_inputs(lens, Hq, Hkv, d, page, seed=1234, dev="cuda"):
 def run(a) -> dict:
     tik.load()
     dev = "cuda"
-    flush = None if a.no_flush else torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    flush = None if a.no_flush else L2Flush(dev, read_pass=not a.write_only_flush)
     scale = float(np.float32(1.0 / np.sqrt(a.d)))
     out = {"case": a.case, "flush": not a.no_flush}
     if a.case == "train":
@@ -146,6 +162,7 @@ def main(argv=None):
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--write-only-flush", action="store_true", help="L2 flush without the read pass (dirty L2)")
     a = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("microbench needs a CUDA device: the library has no CPU path")
