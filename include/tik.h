@@ -177,6 +177,19 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse,
                             int page_size, int num_pages, float softmax_scale, void* ws,
                             size_t ws_bytes, void* stream);
 
+/* Cache write and prefill in one call (paper Sec. 4.1: prefill both fills the KV cache and scores
+ * the prompt): tik_kv_cache_write of the new tokens' keys and values followed by tik_attn_prefill
+ * of their queries, on the same stream.  The new tokens are the query tokens: row i of k_new / v_new
+ * ([total_q][Hkv][d]) belongs to the same token as row i of q, sequence s owns rows
+ * cu_seqlens_q[s] .. cu_seqlens_q[s+1]-1 at positions ctx_lens[s]-q_len[s] .. ctx_lens[s]-1.
+ * Output bits are those of the two separate calls. */
+tik_status tik_attn_prefill_kv(tik_ctx* ctx, const void* q, const void* k_new, const void* v_new, void* o,
+                               float* lse, const int32_t* cu_seqlens_q, const int32_t* ctx_lens,
+                               void* k_cache, void* v_cache, const int32_t* block_table,
+                               int max_blocks, int S, int64_t total_q, int max_q_len, int max_ctx_len,
+                               int Hq, int Hkv, int d, int page_size, int num_pages,
+                               float softmax_scale, void* ws, size_t ws_bytes, void* stream);
+
 /* Token-wise decode attention (paper Sec. 4.1: the decode entry point): one query token
  * per sequence at position ctx_lens[b]-1 (its own key/value already written) against keys
  * 0..ctx_lens[b]-1.  q, o [B][Hq][d]; lse optional fp32 [B][Hq].  A slot with

@@ -98,7 +98,8 @@ def run_grid(reps: int = 20) -> Dict[str, float]:
     from . import binding as tik
     from . import synth
     Hq, Hkv, d, page = HEADS
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    from .microbench import L2Flush
+    flush = L2Flush("cuda")          # cold and clean L2 before every timed launch
     out: Dict[str, float] = {}
     # one pool holds 16 sequences of 8192 tokens (decode) / one of 16384 (prefill)
     w = synth.custom_workload([16384], [0], Hq, Hkv, d, page, index=70)

@@ -55,6 +55,9 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.tik_kv_cache_write.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, i32, i32, vp]
     lib.tik_attn_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, i32, i32,
                                      i32, i32, i32, f32, vp, sz, vp]
+    lib.tik_attn_prefill_kv.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, i32, i32,
+                                        i32, i32, i32, f32, vp, sz, vp]
+    lib.tik_attn_prefill_kv.restype = i32
     lib.tik_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32,
                                     f32, vp, sz, vp]
     lib.tik_qk_norm_rope_kv_write.argtypes = [vp, vp, vp, vp, vp, vp, f32, vp, i32, vp, vp, vp, vp, vp, i32, i32,
@@ -266,6 +269,27 @@ def tik_attn_prefill(q, cu_seqlens_q, ctx_lens, k_cache, v_cache, block_table, m
                                  block_table.shape[1], ctx_lens.numel(), totq, max_q_len, max_ctx_len,
                                  Hq, Hkv, d, page, num_pages, softmax_scale, _ptr(ws),
                                  ws.numel() if ws is not None else 0, _stream())
+    _check(rc, ctx)
+    return o
+
+
+def tik_attn_prefill_kv(q, k_new, v_new, cu_seqlens_q, ctx_lens, k_cache, v_cache, block_table, max_q_len: int,
+                        max_ctx_len: int, softmax_scale: float, o: Optional[torch.Tensor] = None,
+                        lse: Optional[torch.Tensor] = None, ws=None):
+    """Cache write of k_new / v_new [totq,Hkv,d] and prefill of q [totq,Hq,d] in one call -> o."""
+    ctx = context()
+    bf = torch.bfloat16
+    totq, Hq, d = q.shape
+    num_pages, Hkv, page, _ = k_cache.shape
+    if o is None:
+        o = torch.empty_like(q)
+    ws = _plan_ws(OP_ATTN_PREFILL, ctx_lens.numel(), max_ctx_len, ws, q.device)
+    rc = load().tik_attn_prefill_kv(ctx, _ptr(q, bf), _ptr(k_new, bf), _ptr(v_new, bf), _ptr(o, bf),
+                                    _ptr(lse, torch.float32), _ptr(cu_seqlens_q, torch.int32),
+                                    _ptr(ctx_lens, torch.int32), _ptr(k_cache, bf), _ptr(v_cache, bf),
+                                    _ptr(block_table, torch.int32), block_table.shape[1], ctx_lens.numel(), totq,
+                                    max_q_len, max_ctx_len, Hq, Hkv, d, page, num_pages, softmax_scale, _ptr(ws),
+                                    ws.numel() if ws is not None else 0, _stream())
     _check(rc, ctx)
     return o
 

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libtik.so")
-SOURCES = ["tik_api.cu", "tik_attn.cu", "tik_attn_persist.cu", "tik_logprob.cu", "tik_static.cu", "tik_prep.cu", "tik_ffn.cu", "tik_linear.cu", "tik_attn_bwd.cu"]
+SOURCES = ["tik_api.cu", "tik_attn.cu", "tik_attn_persist.cu", "tik_decode.cu", "tik_logprob.cu", "tik_static.cu", "tik_prep.cu", "tik_ffn.cu", "tik_linear.cu", "tik_attn_bwd.cu"]
 HEADERS = ["tik_core.cuh", "tik_ptx.cuh", "tik_internal.h", os.path.join("..", "..", "include", "tik.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]

@@ -333,6 +333,25 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_prefill");
 }
 
+tik_status tik_attn_prefill_kv(tik_ctx* ctx, const void* q, const void* k_new, const void* v_new, void* o,
+                               float* lse, const int32_t* cu_seqlens_q, const int32_t* ctx_lens, void* k_cache,
+                               void* v_cache, const int32_t* block_table, int max_blocks, int S, int64_t total_q,
+                               int max_q_len, int max_ctx_len, int Hq, int Hkv, int d, int page_size,
+                               int num_pages, float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
+    // argument checks of both halves run before anything is queued: a refused call writes nothing
+    if (!ctx) return TIK_ERR_INVALID_ARG;
+    tik_status s = check_heads(ctx, Hq, Hkv, d, softmax_scale);
+    if (s != TIK_OK) return s;
+    if (S > 0 && total_q > 0 && (!q || !o)) return fail(ctx, TIK_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(q) || !aligned16(o)) return fail(ctx, TIK_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    s = tik_kv_cache_write(ctx, k_new, v_new, cu_seqlens_q, ctx_lens, k_cache, v_cache, block_table, max_blocks, S,
+                           total_q, Hkv, d, page_size, num_pages, stream);
+    if (s != TIK_OK) return s;
+    return tik_attn_prefill(ctx, q, o, lse, cu_seqlens_q, ctx_lens, k_cache, v_cache, block_table, max_blocks, S,
+                            total_q, max_q_len, max_ctx_len, Hq, Hkv, d, page_size, num_pages, softmax_scale, ws,
+                            ws_bytes, stream);
+}
+
 tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, const int32_t* ctx_lens,
                            const void* k_cache, const void* v_cache, const int32_t* block_table, int max_blocks,
                            int B, int max_ctx_len, int Hq, int Hkv, int d, int page_size, int num_pages,
@@ -382,12 +401,19 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     p.part_o = static_cast<float*>(ws);
     p.part_ml = p.part_o + static_cast<size_t>(B) * Hq * nchunk * d;
     p.dev_status = ctx->dev_status;
-    p.cpc = decode_chunks_per_cta(B, Hkv, nchunk, ctx->sm_count);
+    // Two kernels give the same bits.  With few (sequence, KV head) pairs -- at most one per SM -- the
+    // small CTA of tik_decode.cu (two per SM, every chunk resident at once) wins: the one-CTA-per-SM
+    // kernel leaves SMs idle or runs a ragged second wave.  With more pairs that kernel's deeper
+    // per-CTA pipeline (two softmax warpgroups, five K/V stages) streams faster per SM, which is
+    // what counts once every SM has several CTAs to run (measured on B200, both at full and at
+    // power-capped clocks).
+    const bool small_group = G <= DECODE2_MAX_G && static_cast<long long>(B) * Hkv <= ctx->sm_count;
+    p.cpc = decode_chunks_per_cta(B, Hkv, nchunk, ctx->sm_count, small_group ? 2 : 1);
     p.lookahead = ctx->sm_count;
     dim3 grid((nchunk + p.cpc - 1) / p.cpc, Hkv, B);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hkv and B must be <= 65535");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_attn(d, 2, grid, tmQ, tmK, tmV, p, st);
+    cudaError_t e = small_group ? launch_decode2(d, grid, tmQ, tmK, tmV, p, st) : launch_attn(d, 2, grid, tmQ, tmK, tmV, p, st);
     if (e == cudaSuccess) e = launch_combine(d, p, B, st);
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_decode");
 }

@@ -76,6 +76,11 @@ struct AttnParams {
 cudaError_t launch_attn(int d, int mode, dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                         const CUtensorMap& tmV, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_combine(int d, const AttnParams& p, int B, cudaStream_t stream);
+// Decode for query groups of at most DECODE2_MAX_G heads (tik_decode.cu): two small CTAs per SM,
+// same grid, scratch layout and output bits as launch_attn in decode mode.
+constexpr int DECODE2_MAX_G = 8;
+cudaError_t launch_decode2(int d, dim3 grid, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                           const AttnParams& p, cudaStream_t stream);
 
 // Persistent full-sequence attention (tik_attn_persist.cu): a planning kernel writes the list of
 // work items of the call into `plan` (attn_plan_bytes bytes, 16-byte aligned), then one CTA per SM
@@ -109,11 +114,16 @@ cudaError_t launch_prep(int d, const PrepParams& p, int64_t total_new, cudaStrea
 
 // Decode: how many consecutive chunks one CTA streams.  A CTA's set-up and drain cost about a
 // third of one chunk's streaming time, so several chunks per CTA pay as long as the grid still
-// covers every SM several times over.  Chunk partials do not depend on this choice.
-inline int decode_chunks_per_cta(long long B, int Hkv, int nchunk, int sm_count) {
-    const long long want = 4ll * (sm_count > 0 ? sm_count : 148);
+// covers every CTA slot several times over.  Chunk partials do not depend on this choice.
+// With two resident CTAs per SM (tik_decode.cu) a CTA's rate is bound by its own serial chain and
+// short ring (measured ~22 GB/s per CTA), so what counts is that all slots stay busy and that no
+// CTA is long: many one-chunk CTAs that the hardware deals out dynamically do that better than few
+// long ones (a batch of ragged contexts is as slow as its longest CTA).  Chunks are grouped only
+// when the grid stays above four waves.
+inline int decode_chunks_per_cta(long long B, int Hkv, int nchunk, int sm_count, int ctas_per_sm = 1) {
+    const long long slots = static_cast<long long>(ctas_per_sm) * (sm_count > 0 ? sm_count : 148);
     for (int c = 4; c > 1; --c)
-        if (c <= nchunk && B * Hkv * ((nchunk + c - 1) / c) >= want) return c;
+        if (c <= nchunk && B * Hkv * ((nchunk + c - 1) / c) >= 4 * slots) return c;
     return 1;
 }
 cudaError_t launch_kv_write(const void* k_new, const void* v_new, const int32_t* cu_new,

@@ -33,6 +33,7 @@ struct DeviceSetup {
     void* scratch = nullptr;     // device address of g_static_scratch on this device
     int* flags = nullptr;        // device address of g_static_flags on this device
     void* encode_tiled = nullptr;
+    int sm_count = 0;
 };
 DeviceSetup g_setup[kMaxDevices];
 std::mutex g_setup_mutex;
@@ -57,6 +58,7 @@ cudaError_t setup_device(int device, DeviceSetup** out) {
         s.scratch = scratch;
         s.flags = static_cast<int*>(flags);
         s.encode_tiled = fn;
+        if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) s.sm_count = 0;
         s.ready = true;
     }
     *out = &s;
@@ -142,7 +144,9 @@ extern "C" tik_status tik_attn_decode_static(const void* q, void* o, float* lse,
     // make every later kernel bail out, so it is cleared (stream-ordered) before each use.
     if (!dev_flags) e = cudaMemsetAsync(s->flags, 0, sizeof(int), st);
     p.cpc = 1;
-    if (e == cudaSuccess) e = launch_attn(d, 2, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st);
+    if (e == cudaSuccess)
+        e = (G <= DECODE2_MAX_G && B * Hkv <= s->sm_count) ? launch_decode2(d, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st)
+                               : launch_attn(d, 2, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st);
     if (e == cudaSuccess) e = launch_combine(d, p, B, st);
     return e == cudaSuccess ? TIK_OK : TIK_ERR_CUDA;
 }

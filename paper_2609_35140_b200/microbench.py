@@ -90,7 +90,8 @@ def run(a) -> dict:
         w = synth.custom_workload([1] * len(lens), [L - 1 for L in lens], a.hq, a.hkv, a.d, a.page)
         q, k, v, cu = synth.make_qkv(w, dev)
         o = torch.empty_like(q)
-        med, mn = _time(lambda: tik.tik_attn_train_fwd(q, k, v, cu, max(lens), scale, o=o), a.reps, a.warmup, flush)
+        wsarg = False if a.per_item else None
+        med, mn = _time(lambda: tik.tik_attn_train_fwd(q, k, v, cu, max(lens), scale, o=o, ws=wsarg), a.reps, a.warmup, flush)
         fl = w.train_flops()
         out.update(shape={"lens": lens if len(lens) <= 8 else "%d x ..." % len(lens), "Hq": a.hq, "Hkv": a.hkv, "d": a.d},
                    flops=fl, tflops=fl / (med * 1e-3) / 1e12, tflops_best=fl / (mn * 1e-3) / 1e12)
@@ -101,7 +102,8 @@ def run(a) -> dict:
         o = torch.empty_like(q)
         cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device=dev)
         ctx = torch.tensor(lens, dtype=torch.int32, device=dev)
-        med, mn = _time(lambda: tik.tik_attn_prefill(q, cu, ctx, kc, vc, bt, max(lens), max(lens), scale, o=o),
+        wsarg = False if a.per_item else None
+        med, mn = _time(lambda: tik.tik_attn_prefill(q, cu, ctx, kc, vc, bt, max(lens), max(lens), scale, o=o, ws=wsarg),
                         a.reps, a.warmup, flush)
         fl = 4.0 * a.d * a.hq * sum(L * (L + 1) // 2 for L in lens)
         out.update(shape={"prompts": len(lens), "len": max(lens), "Hq": a.hq, "Hkv": a.hkv, "d": a.d, "page": a.page},
@@ -162,6 +164,7 @@ def main(argv=None):
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--per-item", action="store_true", help="train / prefill without scratch: one CTA per work item")
     ap.add_argument("--write-only-flush", action="store_true", help="L2 flush without the read pass (dirty L2)")
     a = ap.parse_args(argv)
     if not torch.cuda.is_available():

@@ -160,3 +160,26 @@ def test_decode_context_above_the_host_bound_is_cut_and_flagged(tik):
     assert flags == tik.DEV_BAD_CONTEXT
     assert count_diff(out, ref) == 0                          # slot 1 cut to the bound, slots 0 and 2 untouched by it
     assert bool((ws[need:] == 0x5A).all())
+
+
+def test_prefill_kv_equals_cache_write_then_prefill(tik):
+    """The one-call form leaves the same cache and the same output bits as the two calls, also for a
+    second chunk behind a cached prefix."""
+    w = synth.custom_workload([300, 1100, 64], [1, 1, 1], 8, 2, 128, 64)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    layout = synth.make_paged_layout(w)
+    ro = Rollout(tik, w, q, k, v, layout)
+    cu_h = w.cu_seqlens()
+    kc = torch.zeros_like(ro.kc)
+    vc = torch.zeros_like(ro.vc)
+    for a, b in (([0, 0, 0], [170, 1000, 64]), ([170, 1000, 64], [300, 1100, 64])):
+        rows, o_ref = ro.prefill(start=a, stop=b)
+        lens = [y - x for x, y in zip(a, b)]
+        if max(lens) == 0:
+            continue
+        cu_q = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+        ctx = torch.tensor(b, dtype=torch.int32, device="cuda")
+        o = tik.tik_attn_prefill_kv(q[rows].contiguous(), k[rows].contiguous(), v[rows].contiguous(), cu_q, ctx, kc, vc,
+                                    ro.bt, max(lens), max(b), w.softmax_scale)
+        assert count_diff(o, o_ref) == 0
+        assert torch.equal(bits(kc), bits(ro.kc)) and torch.equal(bits(vc), bits(ro.vc))
