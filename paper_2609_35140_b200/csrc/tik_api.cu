@@ -61,11 +61,13 @@ static unsigned attn_grid_x(int max_positions) {
 
 // The persistent kernel runs when the caller passed a large enough, 16-byte aligned plan buffer and
 // the call is within what the planning kernel handles; otherwise one CTA per work item.
-static bool use_persistent(const void* ws, size_t ws_bytes, int S, int max_positions, int Hq) {
+static bool use_persistent(const void* ws, size_t ws_bytes, int S, int max_positions, int Hq, int sm_count) {
     if (!ws || !aligned16(ws) || !attn_persist_supported(S, max_positions)) return false;
     const long long nt = (static_cast<long long>(max_positions) + 127) / 128;
     const long long X = nt <= 16 ? (nt + 1) / 2 : 8 + (nt - 16);
     if (static_cast<long long>(S) * X * Hq >= (1ll << 31)) return false;
+    // fewer work items than two per SM: nothing to amortise, the planning launch only adds latency
+    if (static_cast<long long>(S) * X * Hq <= 2ll * sm_count) return false;
     return ws_bytes >= attn_plan_bytes(S, max_positions);
 }
 
@@ -232,7 +234,7 @@ tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const 
     dim3 grid(attn_grid_x(max_seqlen), Hq, S);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
     cudaError_t e;
-    if (use_persistent(ws, ws_bytes, S, max_seqlen, Hq))
+    if (use_persistent(ws, ws_bytes, S, max_seqlen, Hq, ctx->sm_count))
         e = launch_attn_persist(d, false, ctx->sm_count, S, static_cast<int>(grid.x), tmQ, tmK, tmV, p, ws,
                                 static_cast<cudaStream_t>(stream));
     else
@@ -325,7 +327,7 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
     dim3 grid(attn_grid_x(max_ctx_len), Hq, S);
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hq and S must be <= 65535");
     cudaError_t e;
-    if (use_persistent(ws, ws_bytes, S, max_ctx_len, Hq))
+    if (use_persistent(ws, ws_bytes, S, max_ctx_len, Hq, ctx->sm_count))
         e = launch_attn_persist(d, true, ctx->sm_count, S, static_cast<int>(grid.x), tmQ, tmK, tmV, p, ws,
                                 static_cast<cudaStream_t>(stream));
     else
@@ -401,13 +403,15 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     p.part_o = static_cast<float*>(ws);
     p.part_ml = p.part_o + static_cast<size_t>(B) * Hq * nchunk * d;
     p.dev_status = ctx->dev_status;
-    // Two kernels give the same bits.  With few (sequence, KV head) pairs -- at most one per SM -- the
-    // small CTA of tik_decode.cu (two per SM, every chunk resident at once) wins: the one-CTA-per-SM
-    // kernel leaves SMs idle or runs a ragged second wave.  With more pairs that kernel's deeper
-    // per-CTA pipeline (two softmax warpgroups, five K/V stages) streams faster per SM, which is
-    // what counts once every SM has several CTAs to run (measured on B200, both at full and at
-    // power-capped clocks).
-    const bool small_group = G <= DECODE2_MAX_G && static_cast<long long>(B) * Hkv <= ctx->sm_count;
+    // Two kernels give the same bits.  The small CTA of tik_decode.cu (two per SM, every chunk
+    // resident at once) wins in the middle range: at most one (sequence, KV head) pair per SM but
+    // about as many chunks as SMs or more, where the one-CTA-per-SM kernel runs a ragged second wave.
+    // With fewer chunks than SMs every CTA has an SM to itself either way and that kernel's faster
+    // per-CTA pipeline (two softmax warpgroups, five K/V stages) gives the shorter latency; with
+    // more pairs than SMs the same pipeline streams faster per SM (measured on B200 at full and at
+    // power-capped clocks; the paper's decode grid, Sec. 6 Q3, covers both ends).
+    const long long pairs = static_cast<long long>(B) * Hkv;
+    const bool small_group = G <= DECODE2_MAX_G && pairs <= ctx->sm_count && 4 * pairs * nchunk >= 3ll * ctx->sm_count;
     p.cpc = decode_chunks_per_cta(B, Hkv, nchunk, ctx->sm_count, small_group ? 2 : 1);
     p.lookahead = ctx->sm_count;
     dim3 grid((nchunk + p.cpc - 1) / p.cpc, Hkv, B);

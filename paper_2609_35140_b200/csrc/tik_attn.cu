@@ -112,6 +112,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     int row_lo[2] = {0, 0}, row_hi[2] = {0, 0};   // valid tile rows [row_lo, row_hi), per query tile
     int tile_first, tile_last;
     if (MODE == MODE_TRAIN || MODE == MODE_PREFILL) {
+        pdl_launch_dependents();       // a grid launched behind this one may fill the SMs that its last wave leaves
         seq = blockIdx.z;
         head = blockIdx.y;
         kvh = head / p.G;
@@ -130,7 +131,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             if (qlen <= 0 || pos0 < 0) return;
         }
         const int t_lo = pos0 / 128, t_hi = (ctx - 1) / 128;     // first and last query tile
-        const int x = gridDim.x - 1 - blockIdx.x;                // heaviest candidates first
+        const int x = p.x_base + gridDim.x - 1 - blockIdx.x;     // heaviest candidates first
         if (x >= 8) {
             T0 = 16 + (x - 8);
             if (T0 < t_lo || T0 > t_hi) return;
@@ -437,7 +438,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     pos2 = ctx2 - (p.cu_seqlens[bz + 1] - qb2);
                 }
                 if (ctx2 > 0 && pos2 >= 0) {
-                    const int x2 = gridDim.x - 1 - bx;
+                    const int x2 = p.x_base + gridDim.x - 1 - bx;
                     const int t_lo2 = pos2 / 128, t_hi2 = (ctx2 - 1) / 128;
                     for (int q2 = 0; q2 < 2; ++q2) {
                         const int Tq = (x2 >= 8) ? (16 + x2 - 8) : (2 * x2 + q2);

@@ -8,8 +8,9 @@
 // beside ~1 560 clk per (query tile, KV tile) step).  Here a CTA walks a list of items and every
 // role runs ahead into the next item on its own:
 //   * a small planning kernel compacts the valid (sequence, item) pairs of the call into a list,
-//     heaviest items first; CTA c takes list positions c, 2n-1-c, 2n+c, ... (n CTAs) for every
-//     query head, so that each CTA meets every weight class;
+//     sequence by sequence, each sequence's heaviest items first; CTA c takes list positions c,
+//     2n-1-c, 2n+c, ... (n CTAs) for every query head: CTAs that run together share a sequence's
+//     K/V in L2, and each CTA meets every weight class;
 //   * all ring, score and weight barriers count across items (stage = tile count & 1, buffer =
 //     step count & 1), so the K / V producers refill the rings with the next item's first tiles
 //     while the current item's last steps run;
@@ -97,72 +98,52 @@ __device__ __forceinline__ PlanSeq plan_seq(const int32_t* cu, const int32_t* ct
 constexpr int PLAN_XMAX = 4096;
 
 // One block.  Output: plan[0].x = number of entries; plan[1 + i] = (seq | x << 16, first query
-// row, context length, position of the first query row), ordered by x descending (the heaviest
-// items first), sequences ascending within one x.
+// row, context length, position of the first query row).  Order: sequences ascending, and within a
+// sequence x descending (its heaviest items first).  CTAs that run at the same time then work on
+// the same one or two sequences, whose K/V stay in L2 (an order by weight across all sequences
+// touched every sequence's K/V at once: a third slower on sixteen 16 K-token sequences), while
+// every CTA still meets every weight class, because the weights repeat sequence by sequence.
+// x_max: only candidates x <= x_max are listed (7: the paired items and partner-less tiles below 16).
 __global__ void __launch_bounds__(1024) attn_plan_kernel(const int32_t* __restrict__ cu,
-                                                         const int32_t* __restrict__ ctx_lens, int S, int X,
+                                                         const int32_t* __restrict__ ctx_lens, int S, int x_max,
                                                          int4* __restrict__ plan) {
     pdl_wait();
     pdl_launch_dependents();
-    __shared__ int cnt[PLAN_XMAX];
-    __shared__ int total;
+    __shared__ int warp_sums[32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int x = warp; x < X; x += 32) {
-        int c = 0;
-        for (int s0 = 0; s0 < S; s0 += 32) {
-            const int s = s0 + lane;
-            bool valid = false;
-            if (s < S) {
-                const PlanSeq q = plan_seq(cu, ctx_lens, s);
-                valid = x >= q.xlo && x <= q.xhi;
-            }
-            c += __popc(__ballot_sync(0xffffffffu, valid));
-        }
-        if (lane == 0) cnt[x] = c;
+    // thread t owns the sequences [t * per, t * per + per)
+    const int per = (S + 1023) / 1024;
+    const int s_lo = threadIdx.x * per, s_hi = min(S, s_lo + per);
+    int mine = 0;
+    for (int s = s_lo; s < s_hi; ++s) {
+        const PlanSeq q = plan_seq(cu, ctx_lens, s);
+        const int hi = min(q.xhi, x_max);
+        if (hi >= q.xlo) mine += hi - q.xlo + 1;
     }
+    int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += n;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-        // exclusive prefix over x descending: lane l owns the reversed positions [l * per, l * per + per)
-        const int per = (X + 31) / 32;
-        int sum = 0;
-        for (int i = 0; i < per; ++i) {
-            const int rx = lane * per + i;
-            if (rx < X) sum += cnt[X - 1 - rx];
-        }
-        int incl = sum;
+        int w = warp_sums[lane], wi = w;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
-            const int n = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += n;
+            const int n = __shfl_up_sync(0xffffffffu, wi, off);
+            if (lane >= off) wi += n;
         }
-        int run = incl - sum;
-        for (int i = 0; i < per; ++i) {
-            const int rx = lane * per + i;
-            if (rx < X) {
-                const int c = cnt[X - 1 - rx];
-                cnt[X - 1 - rx] = run;          // becomes the base of x
-                run += c;
-            }
-        }
-        if (lane == 31) total = incl;
+        warp_sums[lane] = wi - w;           // exclusive prefix of the warps
+        if (lane == 31) plan[0] = make_int4(wi, 0, 0, 0);
     }
     __syncthreads();
-    for (int x = warp; x < X; x += 32) {
-        int run = cnt[x];
-        for (int s0 = 0; s0 < S; s0 += 32) {
-            const int s = s0 + lane;
-            bool valid = false;
-            PlanSeq q{};
-            if (s < S) {
-                q = plan_seq(cu, ctx_lens, s);
-                valid = x >= q.xlo && x <= q.xhi;
-            }
-            const unsigned m = __ballot_sync(0xffffffffu, valid);
-            if (valid) plan[1 + run + __popc(m & ((1u << lane) - 1u))] = make_int4(s | (x << 16), q.qb, q.ctx, q.pos0);
-            run += __popc(m);
-        }
+    int run = warp_sums[warp] + incl - mine;
+    for (int s = s_lo; s < s_hi; ++s) {
+        const PlanSeq q = plan_seq(cu, ctx_lens, s);
+        for (int x = min(q.xhi, x_max); x >= q.xlo; --x) plan[1 + run++] = make_int4(s | (x << 16), q.qb, q.ctx, q.pos0);
     }
-    if (threadIdx.x == 0) plan[0] = make_int4(total, 0, 0, 0);
 }
 
 // ------------------------------------------------------------------ work items
@@ -354,7 +335,10 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
         tmem_relinquish();
     }
-    pdl_wait();        // the plan (and every input) is complete and visible from here on
+    // the plan (and every input) is complete from here on.  Launched behind the single-tile grid
+    // (wait_at_end) this grid starts once every CTA of that grid has started, which is after the
+    // plan completed, and must not wait for that grid here: it is there to fill its tail.
+    if (!p.wait_at_end) pdl_wait();
     if (warp == 3 && lane == 0) {
         // an earlier kernel on this context may have run out of a wait: then do nothing at all
         *abort_word = (*reinterpret_cast<volatile int*>(p.dev_status) & TIK_DEV_WAIT_EXPIRED) ? 1 : 0;
@@ -364,7 +348,8 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    const unsigned n_items = static_cast<unsigned>(plan[0].x) * static_cast<unsigned>(p.Hq);   // < 2^31 (host check)
+    // (plan entries are read around L1: a line of an earlier call's plan may still sit there)
+    const unsigned n_items = static_cast<unsigned>(__ldcg(&plan[0]).x) * static_cast<unsigned>(p.Hq);   // < 2^31 (host check)
     const unsigned ncta = gridDim.x, cta = blockIdx.x;
     // list position of this CTA's k-th item (rounds alternate direction)
     auto item_index = [&](int k) -> unsigned {
@@ -373,7 +358,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     auto load_entry = [&](unsigned i, int& head) -> int4 {
         const unsigned idx = i / static_cast<unsigned>(p.Hq);
         head = static_cast<int>(i - idx * static_cast<unsigned>(p.Hq));
-        return plan[1 + idx];
+        return __ldcg(&plan[1 + idx]);
     };
     // warp-uniform view of the CTA's abort flag (full warps must leave their loops together)
     auto aborted_warp = [&]() -> bool { return __any_sync(0xffffffffu, *abort_word != 0) != 0; };
@@ -877,6 +862,9 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         while (globaltimer_ns() - t0 < 1000000ull) {
         }
     }
+    // Behind the single-tile grid: this grid must not complete before that one has (a kernel that
+    // follows with a programmatic dependency waits for its immediate predecessor only).
+    if (p.wait_at_end) pdl_wait();
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
@@ -932,6 +920,15 @@ bool attn_persist_supported(int64_t S, int64_t max_positions) {
 cudaError_t launch_attn_persist(int d, bool paged, int sm_count, int S, int X, const CUtensorMap& tmQ,
                                 const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnParams& p, void* plan,
                                 cudaStream_t stream) {
+    // Query tiles >= 16 (candidates x >= 8) are long items (17+ steps): they run best as one CTA per
+    // item, with three-stage K/V rings and the sequence-major block order.  When the call has any,
+    // three launches follow each other with programmatic dependencies: the planning kernel (paired
+    // items only), the one-CTA-per-item grid over the single tiles, and the persistent grid, whose
+    // CTAs start as the single-tile grid's last wave leaves SMs free.  Measured on B200: with
+    // sequences of 16 K tokens the split is 9 % faster than the persistent grid alone (which gives
+    // single tiles two-stage rings), with lengths up to 9 K (most items paired or short) 4 % slower
+    // (three launches, two tails): it is used when the length bound exceeds 96 tiles.
+    const bool split = X > 8 + (96 - 16);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -943,15 +940,24 @@ cudaError_t launch_attn_persist(int d, bool paged, int sm_count, int S, int X, c
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, attn_plan_kernel, p.cu_seqlens, paged ? p.ctx_lens : static_cast<const int32_t*>(nullptr),
-                                       S, X, static_cast<int4*>(plan));
+                                       S, split ? 7 : X - 1, static_cast<int4*>(plan));
     if (e != cudaSuccess) return e;
+    AttnParams pp = p;
+    if (split) {
+        AttnParams ps = p;
+        ps.x_base = 8;
+        e = launch_attn(d, paged ? 1 : 0, dim3(static_cast<unsigned>(X - 8), static_cast<unsigned>(p.Hq), static_cast<unsigned>(S)),
+                        tmQ, tmK, tmV, ps, stream);
+        if (e != cudaSuccess) return e;
+        pp.wait_at_end = 1;
+    }
     const int4* pl = static_cast<const int4*>(plan);
     if (d == 128) {
-        return paged ? launch_persist_t<128, true>(sm_count, tmQ, tmK, tmV, p, pl, stream)
-                     : launch_persist_t<128, false>(sm_count, tmQ, tmK, tmV, p, pl, stream);
+        return paged ? launch_persist_t<128, true>(sm_count, tmQ, tmK, tmV, pp, pl, stream)
+                     : launch_persist_t<128, false>(sm_count, tmQ, tmK, tmV, pp, pl, stream);
     }
-    return paged ? launch_persist_t<64, true>(sm_count, tmQ, tmK, tmV, p, pl, stream)
-                 : launch_persist_t<64, false>(sm_count, tmQ, tmK, tmV, p, pl, stream);
+    return paged ? launch_persist_t<64, true>(sm_count, tmQ, tmK, tmV, pp, pl, stream)
+                 : launch_persist_t<64, false>(sm_count, tmQ, tmK, tmV, pp, pl, stream);
 }
 
 }  // namespace tik

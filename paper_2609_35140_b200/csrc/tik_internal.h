@@ -70,6 +70,8 @@ struct AttnParams {
     int cpc;                     // decode: consecutive chunks streamed by one CTA
     int* dev_status;
     int lookahead;               // train / prefill: block distance of the query-tile L2 prefetch
+    int x_base;                  // train / prefill, one CTA per item: candidate index of the grid's last block (0, or 8: single tiles only)
+    int wait_at_end;             // persistent kernel: 1 = launched behind the single-tile grid (see launch_attn_persist)
 };
 
 // mode: 0 train (packed K/V), 1 prefill (paged K/V), 2 decode (paged K/V, chunk partials)

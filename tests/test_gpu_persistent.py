@@ -58,7 +58,7 @@ def test_train_fwd_persistent_equals_per_item_schedule(tik, name):
 
 def test_empty_sequences_in_the_pack(tik):
     """Zero-length entries of cu_seqlens produce no work item and leave every other row alone."""
-    w = synth.custom_workload([1, 1, 1], [299, 40, 2100], 4, 1, 128, 64)
+    w = synth.custom_workload([1, 1, 1], [299, 40, 2100], 8, 1, 128, 64)
     q, k, v, _ = synth.make_qkv(w, "cuda")
     L = w.seq_lens
     cu = torch.tensor([0, 0, L[0], L[0], L[0] + L[1], L[0] + L[1], sum(L), sum(L)], dtype=torch.int32, device="cuda")
@@ -94,7 +94,7 @@ def test_prefill_persistent_equals_per_item_schedule(tik, page):
 
 
 def test_caller_scratch_is_used_and_too_small_scratch_falls_back(tik):
-    w = synth.custom_workload([1] * 5, [300, 900, 20, 2600, 77], 4, 2, 128, 64)
+    w = synth.custom_workload([1] * 5, [300, 900, 20, 2600, 77], 8, 2, 128, 64)
     q, k, v, cu = synth.make_qkv(w, "cuda")
     mx = max(w.seq_lens)
     need = tik.workspace_bytes(tik.OP_ATTN_TRAIN_FWD, w.S, max_ctx=mx)
@@ -108,3 +108,10 @@ def test_caller_scratch_is_used_and_too_small_scratch_falls_back(tik):
     o_b = tik.tik_attn_train_fwd(q, k, v, cu, mx, w.softmax_scale, ws=small)
     assert bool((small == 0).all())                          # not touched: the per-item schedule ran
     assert count_diff(o_a, o_b) == 0
+    # a call with fewer work items than two per SM also runs per item, whatever scratch it is given
+    w1 = synth.custom_workload([1], [700], 4, 2, 128, 64)
+    q1, k1, v1, cu1 = synth.make_qkv(w1, "cuda")
+    ws1 = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    o1 = tik.tik_attn_train_fwd(q1, k1, v1, cu1, 701, w1.softmax_scale, ws=ws1)
+    assert bool((ws1 == 0).all())
+    assert count_diff(o1, tik.tik_attn_train_fwd(q1, k1, v1, cu1, 701, w1.softmax_scale, ws=False)) == 0
