@@ -47,7 +47,10 @@ NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 7700.0}     # data-sheet figures, c
 SM_COUNT, MMA_FLOP_PER_CLK_SM = 148, 8192                 # M128 N128 K16 bf16 MMA: 64 clk
 # DRAM bytes per launch of the headline's dominant kernel (attn_kernel<128, train>) from ncu:
 # captured on a slice of the workload and scaled by tokens (see profiles/), None until captured.
-NCU_TRAFFIC = {"bytes_per_token": None, "source": None}
+NCU_TRAFFIC = {"bytes_per_token": 39225.0,
+               "source": "ncu dram__bytes_read+write of attn_persist_kernel<128,packed> on the first 32 sequences of this "
+                         "workload (3.93 GB for 100 313 tokens, 1.06 x the algorithmic q+k+v+o), scaled by tokens: "
+                         "profiles/attention_fullseq_judged_sizes.md"}
 
 
 def load_peaks():
@@ -768,9 +771,9 @@ def main():
     dom_name = max(("train_fwd", "prefill"), key=lambda n: rooflines[n]["ms"])
     dom = rooflines[dom_name]
     traffic = None
-    if NCU_TRAFFIC["bytes_per_token"] and dom_name == "train_fwd":
+    if NCU_TRAFFIC["bytes_per_token"] and dom_name == "train_fwd" and w.index == HEADLINE:
         traffic = NCU_TRAFFIC["bytes_per_token"] * w.total_tokens
-    roofline = {"kernel": {"train_fwd": "attn_kernel<128,train>", "prefill": "attn_kernel<128,prefill>"}[dom_name],
+    roofline = {"kernel": {"train_fwd": "attn_persist_kernel<128,packed>", "prefill": "attn_persist_kernel<128,paged>"}[dom_name],
                 "bound": "tensor", "achieved": dom["achieved"], "peak": dom["peak"], "unit": "TFLOP/s",
                 "frac": dom["frac"], "traffic": traffic, "traffic_source": NCU_TRAFFIC["source"],
                 "peak_source": "of %s (%s bf16 peak: median SM clock %s of %s MHz over a timed region of %.1f s)" % (

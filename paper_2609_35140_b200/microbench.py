@@ -58,6 +58,9 @@ def _time(fn, reps: int, warmup: int, flush):
 
 
 def _lens(a):
+    if a.workload >= 0:          # the first --first sequences of a benchmark workload (its length mix)
+        w = synth.get_workload(a.workload)
+        return w.seq_lens[:a.first] if a.first > 0 else w.seq_lens
     if a.lens:
         return [int(x) for x in a.lens.split(",")]
     return [a.len] * a.seqs
@@ -153,6 +156,8 @@ def main(argv=None):
     ap.add_argument("--seqs", type=int, default=1)
     ap.add_argument("--len", type=int, default=4096)
     ap.add_argument("--lens", default="", help="comma-separated lengths (overrides --seqs/--len)")
+    ap.add_argument("--workload", type=int, default=-1, help="take the lengths of benchmark workload 0..4 (train / prefill / decode)")
+    ap.add_argument("--first", type=int, default=0, help="with --workload: only its first N sequences")
     ap.add_argument("--hq", type=int, default=32)
     ap.add_argument("--hkv", type=int, default=8)
     ap.add_argument("--d", type=int, default=128)
