@@ -69,3 +69,26 @@ def test_static_decode_refuses_problems_beyond_its_scratch():
     assert rc == -3
     torch.cuda.synchronize()
     assert bool((out == 7.0).all())          # nothing was launched
+
+
+def test_static_decode_reports_device_flags_through_the_callers_word():
+    """A block-table entry outside the pool is read as a page of zeros and flagged.  The entry
+    point has no context to keep flags in: they reach the caller only through `dev_flags`."""
+    from paper_2609_35140_b200 import binding as tik
+    tik.load()
+    w, q, ctx, kc, vc, bt = _case(tik, [300, 64], [200, 90], 8, 2, 128, 64, 204)
+    bad = bt.clone()
+    bad[0, 1] = kc.shape[0] + 5
+    ref = tik.tik_attn_decode(q, ctx, kc, vc, bad, max(w.seq_lens), w.softmax_scale)
+    assert tik.device_status() == tik.DEV_BAD_BLOCK          # the context-based entry point keeps it
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.full_like(ref, 7.0)
+    assert tik.tik_attn_decode_static(q, ctx, kc, vc, bad, max(w.seq_lens), w.softmax_scale, out, dev_flags=flags) == 0
+    torch.cuda.synchronize()
+    assert int(flags.item()) == tik.DEV_BAD_BLOCK
+    assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+    assert bool(torch.isfinite(out.float()).all())
+    # without a word the call still succeeds; the flag is discarded (documented in the header)
+    assert tik.tik_attn_decode_static(q, ctx, kc, vc, bad, max(w.seq_lens), w.softmax_scale, out) == 0
+    torch.cuda.synchronize()
+    assert tik.device_status() == 0
