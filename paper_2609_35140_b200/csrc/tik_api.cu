@@ -580,11 +580,17 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     uint64_t st1[1] = {static_cast<uint64_t>(K) * 2};
     uint32_t box[2] = {64, 128};
     const bool pair = T > 128;           // CTA pairs (two-SM MMAs) as soon as there is more than one row tile
-    uint32_t boxB[2] = {64, pair ? 128u : 256u};
+    // one row tile: the decode-shaped schedule (persistent CTAs over column units, only the rows
+    // that exist staged); same MMA chain per output element, so the same bits
+    const bool unit_mode = !pair;
+    const int nu = unit_mode ? linear_unit_cols(N, ctx->sm_count) : 0;
+    const int a_rows = T <= 32 ? 32 : T <= 64 ? 64 : 128;
+    uint32_t boxA[2] = {64, unit_mode ? static_cast<uint32_t>(a_rows) : 128u};
+    uint32_t boxB[2] = {64, unit_mode ? static_cast<uint32_t>(nu) : pair ? 128u : 256u};
     CUtensorMap tmY;
     uint64_t yd[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(T)};
     uint64_t ys[1] = {static_cast<uint64_t>(N) * 2};
-    if (!make_tmap_bf16(ctx, &tmA, x, 2, ad, st1, box, &err) || !make_tmap_bf16(ctx, &tmB, weight, 2, bd, st1, boxB, &err) ||
+    if (!make_tmap_bf16(ctx, &tmA, x, 2, ad, st1, boxA, &err) || !make_tmap_bf16(ctx, &tmB, weight, 2, bd, st1, boxB, &err) ||
         !make_tmap_bf16(ctx, &tmY, y, 2, yd, ys, box, &err))
         return fail(ctx, TIK_ERR_CUDA, err.c_str());
     LinearParams p{};
@@ -600,6 +606,13 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     p.super_cols = 4096;
     while (p.super_cols > 256 && ntile * ((N + p.super_cols - 1) / p.super_cols) < 4ll * ctx->sm_count) p.super_cols /= 2;
     p.nsuper = (N + p.super_cols - 1) / p.super_cols;
+    // two row tiles: the pair kernel, persistent over 256-column steps (decode batches up to 256)
+    const bool pair_units = pair && T <= 256;
+    p.unit_mode = (unit_mode || pair_units) ? 1 : 0;
+    p.nu = nu;
+    p.nunit = unit_mode ? (N + nu - 1) / nu : pair_units ? (N + 255) / 256 : 0;
+    p.a_rows = a_rows;
+    p.sm_count = ctx->sm_count;
     p.dev_status = ctx->dev_status;
     cudaError_t e = launch_linear(tmA, tmB, tmY, p, pair, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_linear");

@@ -169,8 +169,35 @@ struct LinearParams {
     int64_t T;
     int K, N, nsuper;
     int super_cols;              // output columns per CTA: 256 .. 4096 (a power of two)
+    int unit_mode;               // T <= 128: persistent CTAs over column units (tmA box a_rows, tmB box nu rows)
+    int nu, nunit, a_rows;       // unit width 128 / 256, ceil(N / nu), staged x rows 32 / 64 / 128
+    int sm_count;
     int* dev_status;
 };
+// Unit width of the decode-shaped linear kernel.  Cost model per 64-wide K slice of one unit: the
+// slice's W bytes over the CTA's share of memory bandwidth (HBM rate over the active CTAs, at most
+// ~80 GB/s into one SM), but never less than the ~280 ns that four dependent K16 MMAs on one
+// accumulator take whatever their width; a CTA runs `waves` units one after the other.  The
+// cheapest width wins, the wider one on ties (x is staged once per unit).
+inline int linear_unit_cols(int N, int sm_count) {
+    int best = 256;
+    double best_cost = -1.0;
+    for (int nu = 256; nu >= 128; nu /= 2) {   // 64 never wins: its slices sit on the 280 ns floor
+        const long long units = (N + nu - 1) / nu;
+        const long long waves = (units + sm_count - 1) / sm_count;
+        const double active = static_cast<double>(units < sm_count ? units : sm_count);
+        double rate = 6500.0 / active;                 // bytes per ns
+        if (rate > 80.0) rate = 80.0;
+        double slice_ns = nu * 128.0 / rate;
+        if (slice_ns < 280.0) slice_ns = 280.0;
+        const double cost = waves * slice_ns;
+        if (best_cost < 0.0 || cost < best_cost * 0.999) {
+            best_cost = cost;
+            best = nu;
+        }
+    }
+    return best;
+}
 cudaError_t launch_linear(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                           const LinearParams& p, bool pair, cudaStream_t stream);
 
