@@ -222,6 +222,8 @@ tik_status tik_attn_train_fwd(tik_ctx* ctx, const void* q, const void* k, const 
 
     AttnParams p{};
     if (!make_tmap_bf16(ctx, &p.tmO, o, 3, qd, qs, box, &err)) return fail(ctx, TIK_ERR_CUDA, err.c_str());
+    uint32_t box32[3] = {64, 1, 32};
+    if (!make_tmap_bf16(ctx, &p.tmO32, o, 3, qd, qs, box32, &err)) return fail(ctx, TIK_ERR_CUDA, err.c_str());
     p.o = o;
     p.lse = lse;
     p.cu_seqlens = cu_seqlens;
@@ -306,6 +308,8 @@ tik_status tik_attn_prefill(tik_ctx* ctx, const void* q, void* o, float* lse, co
 
     AttnParams p{};
     if (!make_tmap_bf16(ctx, &p.tmO, o, 3, qd, qs, box, &err)) return fail(ctx, TIK_ERR_CUDA, err.c_str());
+    uint32_t box32[3] = {64, 1, 32};
+    if (!make_tmap_bf16(ctx, &p.tmO32, o, 3, qd, qs, box32, &err)) return fail(ctx, TIK_ERR_CUDA, err.c_str());
     p.o = o;
     p.lse = lse;
     p.cu_seqlens = cu_seqlens_q;

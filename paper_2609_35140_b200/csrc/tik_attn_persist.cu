@@ -217,10 +217,18 @@ __device__ __noinline__ void pa_fold_o_tmem(uint32_t t_a, uint32_t t_b, FoldCoef
 template <int NCOLS>
 __device__ __noinline__ void pa_store_rows(uint32_t acc, float inv, int row0, int lo, int hi, int head, int col0, int D,
                                            uint8_t* stage, __nv_bfloat16* o, int Hq, uint32_t odrain_bar,
-                                           uint32_t odrain_n, int lane, int quarter, long long* tr = nullptr) {
+                                           uint32_t odrain_n, int lane, int quarter, const CUtensorMap* tmo,
+                                           long long* tr = nullptr) {
     constexpr int PASS = NCOLS < 64 ? NCOLS : 64;      // columns per pass
     constexpr int NCH = PASS / 8;                       // 16-byte chunks per row and pass
     constexpr int RPI = 32 / NCH;                       // rows per store instruction
+    // A whole tile (all 128 rows belong to the item) with 128-byte staging rows leaves through one
+    // tiled bulk store of 32 rows x 64 columns per warp and pass: the staging layout is the 128-byte
+    // swizzle of the copy engine, lane 0 owns the warp's bulk groups, and the warp goes on as soon
+    // as the store is issued.  The staging buffer is written again only after lane 0 has seen the
+    // previous group's read of it complete -- for the second pass that wait hides behind the pass's
+    // own accumulator load and packing.
+    const bool bulk = PASS == 64 && tmo != nullptr && lo <= 0 && hi >= 128;
 #pragma unroll 1
     for (int a = 0; a < NCOLS / PASS; ++a) {
         uint32_t v[PASS];
@@ -234,6 +242,28 @@ __device__ __noinline__ void pa_store_rows(uint32_t acc, float inv, int row0, in
             __syncwarp();
             if (lane == 0) mbar_arrive_n(odrain_bar, odrain_n);
         }
+        if (bulk) {
+            uint32_t w[PASS / 2];
+#pragma unroll
+            for (int i = 0; i < PASS / 2; ++i)
+                w[i] = pack_bf16x2(finalize_o(__uint_as_float(v[2 * i]), inv), finalize_o(__uint_as_float(v[2 * i + 1]), inv));
+            if (lane == 0) tma_store_wait_read();
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < NCH; ++i)
+                *reinterpret_cast<uint4*>(stage + lane * 128 + ((i ^ (lane & 7)) << 4)) =
+                    make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_3d(tmo, smem_u32(stage), col0 + PASS * a, head, row0 + 32 * quarter);
+                tma_store_commit();
+            }
+            if (tr) tr[3 * a + 1] = tr[3 * a + 2] = clock64();
+            continue;
+        }
+        if (lane == 0) tma_store_wait_read();       // an earlier whole tile may still be leaving the buffer
+        __syncwarp();
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
             uint32_t w4[4];
@@ -695,7 +725,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     long long* tr = nullptr;
 #endif
                     pa_store_rows<D>(to, inv, e_row0, e_lo, e_hi, e_head, 0, D, stage_warp, o_base, p.Hq,
-                                     bar_odrain + 8 * wg, 2u, lane, quarter, tr);
+                                     bar_odrain + 8 * wg, 2u, lane, quarter, &p.tmO32, tr);
                 }
                 if (quarter == 0 && lane == 0) PA_STAMP(k, 17 + 10 * wg);
             } else {
@@ -840,12 +870,13 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     const float inv = st_inv_all[128 * (k & 1) + r];
                     volatile int* m = meta_single + 4 * (k & 1);
                     pa_store_rows<DH>(tlane + COL_OA + DH * wg, inv, m[0], m[1], m[2], m[3], DH * wg, D, stage_warp, o_base,
-                                      p.Hq, bar_odrain, 1u, lane, quarter);
+                                      p.Hq, bar_odrain, 1u, lane, quarter, &p.tmO32);
                 }
                 hc0 += n_tiles;
             }
             Gs0 += n_steps;
         }
+        if (lane == 0) tma_store_wait_all();     // this warp's bulk stores are complete before the CTA ends
     }
     }
 

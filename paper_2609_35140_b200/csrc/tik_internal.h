@@ -53,6 +53,7 @@ bool make_tmap_bf16(tik_ctx* ctx, CUtensorMap* out, const void* base, int rank,
 
 struct AttnParams {
     alignas(64) CUtensorMap tmO; // train / prefill: tiled map of the output (same shape and box as Q)
+    alignas(64) CUtensorMap tmO32;   // the same tensor with a box of 32 rows (persistent kernel: one warp's rows)
     void* o;                     // bf16 output rows
     float* lse;                  // optional
     const int32_t* cu_seqlens;   // train: per sequence; prefill: per sequence, query tokens
