@@ -515,7 +515,7 @@ def time_ffn(hp: "HotPath", peaks, tpeak, reps: int = 5):
     ad, od = act[:xd.shape[0]].contiguous(), torch.empty(xd.shape[0], H, dtype=torch.bfloat16, device="cuda")
     r["linear_down_decode_shaped"] = hbm(time_alone(hp, lambda: tik.tik_linear(ad, w_d, y=od), reps), I * H * 2,
                                          "T=%d rows: weight bytes I*H*2 over the launch time; the fixed K chain of "
-                                         "I/16 dependent MMAs sets a floor of ~4.4 ns per element of I" % xd.shape[0])
+                                         "I/16 MMAs per element on at most H/64 CTAs bounds it" % xd.shape[0])
     return r
 
 

@@ -587,8 +587,8 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     // one row tile: the decode-shaped schedule (persistent CTAs over column units, only the rows
     // that exist staged); same MMA chain per output element, so the same bits
     const bool unit_mode = !pair;
-    const int nu = unit_mode ? linear_unit_cols(N, ctx->sm_count) : 0;
     const int a_rows = T <= 32 ? 32 : T <= 64 ? 64 : 128;
+    const int nu = unit_mode ? linear_unit_cols(N, a_rows, ctx->sm_count) : 0;
     uint32_t boxA[2] = {64, unit_mode ? static_cast<uint32_t>(a_rows) : 128u};
     uint32_t boxB[2] = {64, unit_mode ? static_cast<uint32_t>(nu) : pair ? 128u : 256u};
     CUtensorMap tmY;

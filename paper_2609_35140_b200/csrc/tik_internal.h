@@ -171,26 +171,31 @@ struct LinearParams {
     int K, N, nsuper;
     int super_cols;              // output columns per CTA: 256 .. 4096 (a power of two)
     int unit_mode;               // T <= 128: persistent CTAs over column units (tmA box a_rows, tmB box nu rows)
-    int nu, nunit, a_rows;       // unit width 128 / 256, ceil(N / nu), staged x rows 32 / 64 / 128
+    int nu, nunit, a_rows;       // unit width 64 / 128 / 256, ceil(N / nu), staged x rows 32 / 64 / 128
     int sm_count;
     int* dev_status;
 };
-// Unit width of the decode-shaped linear kernel.  Cost model per 64-wide K slice of one unit: the
-// slice's W bytes over the CTA's share of memory bandwidth (HBM rate over the active CTAs, at most
-// ~80 GB/s into one SM), but never less than the ~280 ns that four dependent K16 MMAs on one
-// accumulator take whatever their width; a CTA runs `waves` units one after the other.  The
-// cheapest width wins, the wider one on ties (x is staged once per unit).
-inline int linear_unit_cols(int N, int sm_count) {
+// Unit width of the decode-shaped linear kernel, from a cost model of one 64-wide K slice of one
+// unit on a B200: its four MMAs (N = 256: 270 ns, 128: 135 ns, 64: 100 ns -- shared-memory bound) plus
+// the issuing thread's ~170 ns per stage spread over the stage's slices; or the slice's bytes (x
+// rows and W rows) into one SM at ~95 GB/s; or its W bytes at the CTA's share of ~6.5 TB/s -- whichever
+// is longest; a CTA runs `waves` units one after the other.  The cheapest width wins, the wider one
+// on ties (x is staged once per unit).
+inline int linear_unit_cols(int N, int a_rows, int sm_count) {
     int best = 256;
     double best_cost = -1.0;
-    for (int nu = 256; nu >= 128; nu /= 2) {   // 64 never wins: its slices sit on the 280 ns floor
+    for (int nu = 256; nu >= 64; nu /= 2) {
         const long long units = (N + nu - 1) / nu;
         const long long waves = (units + sm_count - 1) / sm_count;
         const double active = static_cast<double>(units < sm_count ? units : sm_count);
-        double rate = 6500.0 / active;                 // bytes per ns
-        if (rate > 80.0) rate = 80.0;
-        double slice_ns = nu * 128.0 / rate;
-        if (slice_ns < 280.0) slice_ns = 280.0;
+        const double mma_ns = nu == 256 ? 270.0 : nu == 128 ? 135.0 : 100.0;
+        int kps = 256 / nu;
+        while (kps > 1 && (192 * 1024) / ((a_rows + nu) * 128 * kps) < 3) kps >>= 1;
+        double slice_ns = mma_ns + 170.0 / kps;
+        const double fill_ns = (a_rows + nu) * 128.0 / 95.0;
+        const double hbm_ns = nu * 128.0 / (6500.0 / active);
+        if (fill_ns > slice_ns) slice_ns = fill_ns;
+        if (hbm_ns > slice_ns) slice_ns = hbm_ns;
         const double cost = waves * slice_ns;
         if (best_cost < 0.0 || cost < best_cost * 0.999) {
             best_cost = cost;

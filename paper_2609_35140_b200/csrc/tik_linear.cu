@@ -241,10 +241,10 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 // Decode-shaped calls (one row tile: T <= 128).  The work is one pass over W at HBM rate, so the
 // schedule is built for bytes in flight and even SM load instead of tensor throughput: the grid is
 // one persistent CTA per SM walking column units u = blockIdx.x, + gridDim.x, ...; a unit is
-// `nu` = 128 or 256 output columns (the host picks the width that fills the last wave best);
+// `nu` = 64, 128 or 256 output columns (the host picks the width from a cost model);
 // only `a_rows` = 32, 64 or 128 rows of x are staged per K slice (the MMA still spans 128 rows: rows
 // past a_rows read whatever the stage holds, their accumulator rows are never stored); the ring
-// has as many stages as fit in 192 KiB (4 .. 9), and the producer runs ahead into the next unit
+// has as many stages as fit in 192 KiB (3 .. 4) of one, two or four K slices each, and the producer runs ahead into the next unit
 // while the epilogue of the last one drains.  An output element is still one chain of K16 MMAs in
 // ascending K into one fp32 accumulator, so its bits equal those of the batched kernel.
 namespace linu {
@@ -264,7 +264,14 @@ linear_unit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nu = p.nu;
     const uint32_t a_bytes = static_cast<uint32_t>(p.a_rows) * 128u;
-    const uint32_t stage_bytes = a_bytes + static_cast<uint32_t>(nu) * 128u;      // a multiple of 1 KiB
+    const uint32_t slice_bytes = a_bytes + static_cast<uint32_t>(nu) * 128u;      // a multiple of 1 KiB
+    // K slices per stage: the issuing thread spends ~300 cycles per stage on its barrier wait, fence,
+    // descriptors and commit, more than four narrow MMAs run (N = 128: 256 cycles, N = 64: ~190);
+    // 256 / nu slices per stage (as long as three stages fit) bring that share down (N = 256 MMAs run
+    // 512 cycles per slice and hide it)
+    int kps = 256 / nu;
+    while (kps > 1 && RING_BYTES / (slice_bytes * static_cast<uint32_t>(kps)) < 3u) kps >>= 1;
+    const uint32_t stage_bytes = slice_bytes * static_cast<uint32_t>(kps);
     const int nst = min(MAX_STAGES, static_cast<int>(RING_BYTES / stage_bytes));
     const int n_my = (p.nunit - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
     const int n_kb = p.K / 64;
@@ -313,13 +320,16 @@ linear_unit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             uint32_t use = 0;                    // how often stage s has been filled before
             for (int i = 0; i < n_my; ++i) {
                 const int col0 = (static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x)) * nu;
-                for (int kb = 0; kb < n_kb; ++kb) {
+                for (int kb = 0; kb < n_kb; kb += kps) {
                     if (*abort_word) break;
                     if (use > 0) mbar_wait(bar_empty + 8 * s, (use - 1) & 1, abort_word, p.dev_status);
-                    const uint32_t dst = sbase + s * stage_bytes;
-                    mbar_expect_tx(bar_full + 8 * s, stage_bytes);
-                    tma_load_2d(dst + a_bytes, &tmB, bar_full + 8 * s, kb * 64, col0);   // W rows past N: zeros
-                    tma_load_2d(dst, &tmA, bar_full + 8 * s, kb * 64, 0);                // x rows past T: zeros
+                    const int ns = min(kps, n_kb - kb);
+                    mbar_expect_tx(bar_full + 8 * s, slice_bytes * static_cast<uint32_t>(ns));
+                    for (int sl = 0; sl < ns; ++sl) {
+                        const uint32_t dst = sbase + s * stage_bytes + sl * slice_bytes;
+                        tma_load_2d(dst + a_bytes, &tmB, bar_full + 8 * s, (kb + sl) * 64, col0);   // W rows past N: zeros
+                        tma_load_2d(dst, &tmA, bar_full + 8 * s, (kb + sl) * 64, 0);                // x rows past T: zeros
+                    }
                     if (++s == nst) {
                         s = 0;
                         ++use;
@@ -337,13 +347,15 @@ linear_unit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 const uint32_t acc_use = i >> 1;
                 if (acc_use > 0) mbar_wait(bar_acc_empty + 8 * buf, (acc_use - 1) & 1, abort_word, p.dev_status);
                 tc_fence_after();
-                for (int kb = 0; kb < n_kb; ++kb) {
+                for (int kb = 0; kb < n_kb; kb += kps) {
                     if (*abort_word) break;
                     mbar_wait(bar_full + 8 * s, use & 1, abort_word, p.dev_status);
                     tc_fence_after();
                     const uint32_t a0 = sbase + s * stage_bytes, b0 = a0 + a_bytes;
-                    mma_ss_chain4(tmem + buf * 256, smem_desc_sw128(a0, 0, 1024), smem_desc_sw128(b0, 0, 1024),
-                                  idesc, kb ? 1u : 0u);
+                    const int ns = min(kps, n_kb - kb);
+                    for (int sl = 0; sl < ns; ++sl)
+                        mma_ss_chain4(tmem + buf * 256, smem_desc_sw128(a0 + sl * slice_bytes, 0, 1024),
+                                      smem_desc_sw128(b0 + sl * slice_bytes, 0, 1024), idesc, (kb + sl) ? 1u : 0u);
                     mma_commit(bar_empty + 8 * s);
                     if (++s == nst) {
                         s = 0;
