@@ -54,7 +54,15 @@ __device__ long long g_pa_trace[PA_TRACE_ITEMS * PA_TRACE_EVENTS];
 #define PA_TAG(site) pa_tag = (site)
 #define PA_AUX(v) pa_aux = static_cast<int>(v)
 __device__ int g_pa_tags[148 * 12 * 2];
+// per-step stamps of the first 8 items of CTA 0: [item][role: 0 QK issuer, 1 PV issuer, 2 / 3 warpgroups][step < 16][event < 8]
+__device__ long long g_pa_steps[8 * 4 * 16 * 8];
+#define PA_SSTAMP(k, role, g, ev)                                                               \
+    do {                                                                                        \
+        if (blockIdx.x == 0 && (k) < 8 && (g) < 16)                                             \
+            g_pa_steps[(((k) * 4 + (role)) * 16 + (g)) * 8 + (ev)] = clock64();                  \
+    } while (0)
 #else
+#define PA_SSTAMP(k, role, g, ev) do { } while (0)
 #define PA_STAMP(k, ev) do { } while (0)
 #define PA_TAG(site) do { } while (0)
 #define PA_AUX(v) do { } while (0)
@@ -520,12 +528,14 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if (g == 0) PA_STAMP(k, 1);
                     PA_WAIT(4, bar_kfull + 8 * st, (kc >> 1) & 1, abort_word, p.dev_status);
                     if (g == 0) PA_STAMP(k, 2);
+                    PA_SSTAMP(k, 0, g, 0);
                     // the single score buffer is free once the softmax of the previous step holds it in registers
                     if (Gs >= 1) PA_WAIT(5, bar_sempty + 8 * ((Gs - 1) & 1), ((Gs - 1) >> 1) & 1, abort_word, p.dev_status);
                     if (g == 0) PA_STAMP(k, 3);
                     if (g == 1) PA_STAMP(k, 4);
                     if (g == it.n_steps - 1) PA_STAMP(k, 5);
                     tc_fence_after();
+                    PA_SSTAMP(k, 0, g, 1);
                     const uint64_t dk = smem_desc_sw128(sK + st * L::TILE, 0, 1024);
                     if (D == 128) mma_ss_chain8_fresh(tmem + COL_S, tileA ? dqA : dqB, dk, IDESC_QK);
                     else mma_ss_chain4_fresh(tmem + COL_S, tileA ? dqA : dqB, dk, IDESC_QK);
@@ -535,6 +545,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     // so is the query slot: A's last step is n_steps - 2, B's (and a single tile's) the last
                     if (g == it.n_steps - 1) mma_commit(bar_qempty + 8 * sB);
                     else if (it.pair && g == it.n_steps - 2) mma_commit(bar_qempty + 8 * (sB ^ 1));
+                    PA_SSTAMP(k, 0, g, 2);
                     ++Gs;
                 }
                 kbase += it.n_tiles;
@@ -564,6 +575,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if (g == 0) PA_STAMP(k, 6);
                     PA_WAIT(6, bar_vfull + 8 * st, (vc >> 1) & 1, abort_word, p.dev_status);
                     if (g == 0) PA_STAMP(k, 7);
+                    PA_SSTAMP(k, 1, g, 0);
                     PA_WAIT(7, bar_pfull + 8 * b, (Gs >> 1) & 1, abort_word, p.dev_status);
                     if (g == 0) PA_STAMP(k, 8);
                     if (g == it.n_steps - 1) PA_STAMP(k, 9);
@@ -575,10 +587,12 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if ((it.pair ? (g < 2) : (g == 0)) && drained > 0)
                         PA_WAIT(8, bar_odrain + 8 * acc, (drained - 1) & 1, abort_word, p.dev_status);
                     tc_fence_after();
+                    PA_SSTAMP(k, 1, g, 1);
                     mma_ts_chain8(tmem + (acc ? COL_OB : COL_OA), tmem + COL_P + 64 * b,
                                   smem_desc_sw128(sV + st * L::TILE, L::ATOM, 1024), IDESC_PV, fresh ? 0u : 1u);
                     mma_commit(bar_pempty + 8 * b);
                     if (!it.pair || (g & 1) || g == it.n_steps - 1) mma_commit(bar_vempty + 8 * st);
+                    PA_SSTAMP(k, 1, g, 2);
                     ++Gs;
                 }
                 vbase += it.n_tiles;
@@ -655,6 +669,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     PA_WAIT(12, bar_sfull + 8 * wg, (Gg >> 1) & 1, abort_word, p.dev_status);
                     if (quarter == 0 && lane == 0 && g == lp) PA_STAMP(k, 11 + 10 * wg);
                     tc_fence_after();
+                    if (quarter == 0 && lane == 0) PA_SSTAMP(k, 2 + wg, g, 0);
                     {
                     const int kmax = qpos_p - 128 * j;              // columns > kmax are masked
                     uint32_t sc[128];
@@ -667,6 +682,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_sempty + 8 * wg);
+                    if (quarter == 0 && lane == 0) PA_SSTAMP(k, 2 + wg, g, 1);
                     if (kmax < 127) {
 #pragma unroll
                         for (int i = 0; i < 128; ++i)
@@ -689,11 +705,14 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     RowSum4 rs_lo, rs_hi;
                     rs_lo.reset();
                     rs_hi.reset();
+                    if (quarter == 0 && lane == 0) PA_SSTAMP(k, 2 + wg, g, 2);
 #pragma unroll
                     for (int i = 0; i < 64; i += 8) softmax_p8(&sc[i], c, neg_mc, rs_lo, &sc[i >> 1]);
+                    if (quarter == 0 && lane == 0) PA_SSTAMP(k, 2 + wg, g, 3);
                     // The PV of this warpgroup's previous step (possibly the previous item's) read its weight
                     // buffer and updated its accumulator: waited for right before the first store.
                     if (Gg >= 2) wait_pv(Gg - 2);
+                    if (quarter == 0 && lane == 0) PA_SSTAMP(k, 2 + wg, g, 4);
                     tmem_st32(tp, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
 #pragma unroll
                     for (int i = 0; i < 64; i += 8) softmax_p8(&sc[64 + i], c, neg_mc, rs_hi, &sc[32 + (i >> 1)]);
@@ -701,11 +720,13 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     l_lo = __fmaf_rn(l_lo, alpha, rs_lo.total());
                     l_hi = __fmaf_rn(l_hi, alpha, rs_hi.total());
                     if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.0f)) pa_rescale_o_tmem<D>(to, alpha);
+                    if (quarter == 0 && lane == 0) PA_SSTAMP(k, 2 + wg, g, 5);
                     tmem_wait_st();
                     }
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_pfull + 8 * wg);
+                    if (quarter == 0 && lane == 0) PA_SSTAMP(k, 2 + wg, g, 6);
                 }
                 // ---- this tile is complete after its last PV: normalise and store its rows
                 if (quarter == 0 && lane == 0) PA_STAMP(k, 12 + 10 * wg);
@@ -929,6 +950,9 @@ static cudaError_t launch_persist_t(int ncta, const CUtensorMap& tmQ, const CUte
 extern "C" int tik_debug_pa_trace(long long* host_out, int n) {
     const int total = PA_TRACE_ITEMS * PA_TRACE_EVENTS;
     return cudaMemcpyFromSymbol(host_out, g_pa_trace, sizeof(long long) * (n < total ? n : total)) == cudaSuccess ? 0 : -1;
+}
+extern "C" int tik_debug_pa_steps(long long* host_out) {
+    return cudaMemcpyFromSymbol(host_out, g_pa_steps, sizeof(long long) * 8 * 4 * 16 * 8) == cudaSuccess ? 0 : -1;
 }
 extern "C" int tik_debug_pa_tags(int* host_out) {
     return cudaMemcpyFromSymbol(host_out, g_pa_tags, sizeof(int) * 148 * 12 * 2) == cudaSuccess ? 0 : -1;
