@@ -511,7 +511,9 @@ def time_ffn(hp: "HotPath", peaks, tpeak, reps: int = 5):
     # decode-sized projection: one token per sequence, the weights are streamed once (HBM-bound)
     xd, yd = x[:min(w.S, 256)].contiguous(), torch.empty(min(w.S, 256), 2 * I, dtype=torch.bfloat16, device="cuda")
     r["linear_gate_up_decode_shaped"] = hbm(time_alone(hp, lambda: tik.tik_linear(xd, w_gu, y=yd), reps), 2 * I * H * 2,
-                                            "T=%d rows: weight bytes 2I*H*2 over the launch time" % xd.shape[0])
+                                            "T=%d rows: weight bytes 2I*H*2 over the launch time%s" % (
+                                                xd.shape[0], "; at 256 rows the call needs as long on the tensor pipes as on HBM "
+                                                "(ridge point), so it follows the SM clock" if xd.shape[0] > 128 else ""))
     ad, od = act[:xd.shape[0]].contiguous(), torch.empty(xd.shape[0], H, dtype=torch.bfloat16, device="cuda")
     r["linear_down_decode_shaped"] = hbm(time_alone(hp, lambda: tik.tik_linear(ad, w_d, y=od), reps), I * H * 2,
                                          "T=%d rows: weight bytes I*H*2 over the launch time; the fixed K chain of "
