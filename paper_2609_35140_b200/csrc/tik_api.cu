@@ -403,6 +403,7 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     p.num_pages = num_pages;
     p.c = scale_to_c(softmax_scale);
     p.nchunk_max = nchunk;
+    p.direct_out = nchunk == 1 ? 1 : 0;     // contexts of at most one chunk: no partials, no combine launch
     p.max_ctx = max_ctx_len;
     p.part_o = static_cast<float*>(ws);
     p.part_ml = p.part_o + static_cast<size_t>(B) * Hq * nchunk * d;
@@ -422,7 +423,7 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     if (grid.y > 65535 || grid.z > 65535) return fail(ctx, TIK_ERR_UNSUPPORTED, "Hkv and B must be <= 65535");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = small_group ? launch_decode2(d, grid, tmQ, tmK, tmV, p, st) : launch_attn(d, 2, grid, tmQ, tmK, tmV, p, st);
-    if (e == cudaSuccess) e = launch_combine(d, p, B, st);
+    if (e == cudaSuccess && !p.direct_out) e = launch_combine(d, p, B, st);
     return e == cudaSuccess ? TIK_OK : cuda_fail(ctx, e, "tik_attn_decode");
 }
 

@@ -672,12 +672,37 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             // tile, accumulator columns half by each warpgroup's warp 0
             if (wg == (last & 1)) {
                 wait_pv(last);
-                if (quarter == 0) write_partial_ml(chunk_of(last), m_own, l_own_lo, l_own_hi);
+                if (quarter == 0 && !p.direct_out) write_partial_ml(chunk_of(last), m_own, l_own_lo, l_own_hi);
                 tc_fence_before();
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
             tc_fence_after();
-            if (quarter == 0) write_partial_o(chunk_of(last), DH * wg, DH);
+            if (quarter == 0 && !p.direct_out) write_partial_o(chunk_of(last), DH * wg, DH);
+            if (quarter == 0 && p.direct_out) {
+                // One chunk per sequence: its state is the global state (the combine would copy it),
+                // so the rows are normalised and stored here, by the combine's own operations; the
+                // row sums of the last tile's owner are in shared memory since its hand-over.
+                const float Ltot = finalize_l(st_l[lane], st_l[128 + lane]);
+                const float inv = finalize_inv(Ltot);
+                const long long orow = static_cast<long long>(seq) * p.Hq + head + r;
+                __nv_bfloat16* const og = reinterpret_cast<__nv_bfloat16*>(p.o) + orow * D + DH * wg;
+                for (int cc = 0; cc < DH / 32; ++cc) {
+                    uint32_t v[32];
+                    tmem_ld32(tlane + COL_OA + DH * wg + 32 * cc, v);
+                    tmem_wait_ld();
+                    if (r < p.G) {
+                        uint4* dst = reinterpret_cast<uint4*>(og + 32 * cc);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            dst[i] = make_uint4(
+                                pack_bf16x2(finalize_o(__uint_as_float(v[8 * i]), inv), finalize_o(__uint_as_float(v[8 * i + 1]), inv)),
+                                pack_bf16x2(finalize_o(__uint_as_float(v[8 * i + 2]), inv), finalize_o(__uint_as_float(v[8 * i + 3]), inv)),
+                                pack_bf16x2(finalize_o(__uint_as_float(v[8 * i + 4]), inv), finalize_o(__uint_as_float(v[8 * i + 5]), inv)),
+                                pack_bf16x2(finalize_o(__uint_as_float(v[8 * i + 6]), inv), finalize_o(__uint_as_float(v[8 * i + 7]), inv)));
+                    }
+                }
+                if (wg == (last & 1) && r < p.G && p.lse) p.lse[orow] = finalize_lse(m_own, Ltot, c);
+            }
         } else if (pair) {
             // ---- paired mode: this warpgroup keeps the rows of one query tile (wg 0: tile B = T0,
             // wg 1: tile A = T1) through all of that tile's KV tiles; nothing is handed over.

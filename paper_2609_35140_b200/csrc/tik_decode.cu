@@ -227,6 +227,31 @@ decode2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         };
         // partial of a finished chunk: (m, l_lo, l_hi) and the accumulator rows of the G heads
         auto write_partial = [&](int chunk_idx) {
+            if (p.direct_out) {
+                // one chunk per sequence: the partial is the result (see the decode mode of attn_kernel)
+                const float Ltot = finalize_l(l_lo, l_hi);
+                const float inv = finalize_inv(Ltot);
+                const long long orow = static_cast<long long>(seq) * p.Hq + head + lane;
+                __nv_bfloat16* const og = reinterpret_cast<__nv_bfloat16*>(p.o) + orow * D;
+#pragma unroll 1
+                for (int cc = 0; cc < D / 32; ++cc) {
+                    uint32_t v[32];
+                    tmem_ld32(tlane + COL_O + 32 * cc, v);
+                    tmem_wait_ld();
+                    if (lane < p.G) {
+                        uint4* dst = reinterpret_cast<uint4*>(og + 32 * cc);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            dst[i] = make_uint4(
+                                pack_bf16x2(finalize_o(__uint_as_float(v[8 * i]), inv), finalize_o(__uint_as_float(v[8 * i + 1]), inv)),
+                                pack_bf16x2(finalize_o(__uint_as_float(v[8 * i + 2]), inv), finalize_o(__uint_as_float(v[8 * i + 3]), inv)),
+                                pack_bf16x2(finalize_o(__uint_as_float(v[8 * i + 4]), inv), finalize_o(__uint_as_float(v[8 * i + 5]), inv)),
+                                pack_bf16x2(finalize_o(__uint_as_float(v[8 * i + 6]), inv), finalize_o(__uint_as_float(v[8 * i + 7]), inv)));
+                    }
+                }
+                if (lane < p.G && p.lse) p.lse[orow] = finalize_lse(m_run, Ltot, c);
+                return;
+            }
             if (lane < p.G) {
                 const long long slot = (static_cast<long long>(seq) * p.Hq + head + lane) * p.nchunk_max + chunk_idx;
                 p.part_ml[4 * slot] = m_run;

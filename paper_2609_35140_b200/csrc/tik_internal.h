@@ -69,6 +69,8 @@ struct AttnParams {
     int nchunk_max;
     int max_ctx;                 // decode: the host's bound on ctx_lens (sized the grid and the scratch)
     int cpc;                     // decode: consecutive chunks streamed by one CTA
+    int direct_out;              // decode: one chunk per sequence by the host's bound -- the chunk's partial is
+                                 // the result, normalised and stored by the decode kernel itself (no combine)
     int* dev_status;
     int lookahead;               // train / prefill: block distance of the query-tile L2 prefetch
     int x_base;                  // train / prefill, one CTA per item: candidate index of the grid's last block (0, or 8: single tiles only)

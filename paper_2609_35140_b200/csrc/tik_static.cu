@@ -132,6 +132,7 @@ extern "C" tik_status tik_attn_decode_static(const void* q, void* o, float* lse,
     p.num_pages = num_pages;
     p.c = softmax_scale * LOG2E_F;
     p.nchunk_max = nchunk;
+    p.direct_out = nchunk == 1 ? 1 : 0;
     p.max_ctx = max_ctx_len;
     // Every chunk partial that the combine kernel reads is written by the decode kernel of
     // this same call first, so stale contents of the shared scratch are never consumed.
@@ -147,6 +148,6 @@ extern "C" tik_status tik_attn_decode_static(const void* q, void* o, float* lse,
     if (e == cudaSuccess)
         e = (G <= DECODE2_MAX_G && B * Hkv <= s->sm_count && 4ll * B * Hkv * nchunk >= 3ll * s->sm_count) ? launch_decode2(d, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st)
                                : launch_attn(d, 2, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st);
-    if (e == cudaSuccess) e = launch_combine(d, p, B, st);
+    if (e == cudaSuccess && !p.direct_out) e = launch_combine(d, p, B, st);
     return e == cudaSuccess ? TIK_OK : TIK_ERR_CUDA;
 }
