@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the kernels use:
-// mbarrier, TMA tiled loads (never multicast), tcgen05 MMA / TMEM, proxy fences.
+// mbarrier, TMA tiled loads (each CTA fetches its own tiles), tcgen05 MMA / TMEM, proxy fences.
 // Every wait is bounded: after TIK_WAIT_LIMIT_NS the waiter raises a flag in the
 // device status word and in a CTA-local abort word, and every later wait of that
 // CTA returns at once, so a scheduling bug ends the kernel instead of hanging it.
@@ -96,7 +96,7 @@ __device__ __forceinline__ void tc_fence_after() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
-// ---------------------------------------------------------------- TMA (tiled loads, no multicast)
+// ---------------------------------------------------------------- TMA (tiled loads, one destination CTA each)
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
