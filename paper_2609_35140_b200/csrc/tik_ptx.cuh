@@ -372,7 +372,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA tile load into this CTA's shared memory whose bytes are counted on a barrier that may live
-// in the peer CTA (no multicast: every CTA fetches its own tile)
+// in the peer CTA (every CTA fetches its own tile)
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster_addr,
                                                  int c0, int c1) {
     asm volatile(
