@@ -268,6 +268,9 @@ def time_steps(hp: HotPath, steps: int, warmup: int):
     return phase, total_ms
 
 
+ALONE_PAUSE_S = 1.0      # idle time between the timed steps and the phases timed on their own
+
+
 def time_alone(hp: HotPath, fn, reps: int, warmup: int = 2):
     """Median ms of `fn` launched on its own: (L2 flush, event, fn, event) x reps queued back to
     back and synchronised once, so the host's share of a call hides behind the previous flush."""
@@ -593,6 +596,8 @@ def workload_config(w: synth.Workload, n_gpus: int):
             "decode_contexts": w.decode_contexts or "full sequence lengths",
             "l2": "before every phase a 512 MiB buffer is overwritten (L2 flush) and a 256 MiB buffer is read (pushes the "
                   "flush's own dirty lines out, so the phase does not pay for their write-back); excluded from the phase times",
+            "alone": "the phases timed on their own follow the steps after %.0f s of idle time (the step's "
+                     "power state has decayed); they are context for the in-step figures, not part of `value`" % ALONE_PAUSE_S,
             "parallelism": "replicas x%d (no collective)" % n_gpus}
 
 
@@ -612,6 +617,8 @@ def measure_workload(tik, w, steps, warmup, rank, local_rank, headline: bool, wa
     # every attention phase once more on its own (short bursts: the clocks are not held down by the
     # log-prob GEMM of the same step), and the decode-shaped log-prob call (one row per sequence)
     reps = max(3, min(steps, 10))
+    torch.cuda.synchronize()
+    time.sleep(ALONE_PAUSE_S)          # the power state of the steps decays before the short bursts are timed
     nums["alone_train"] = time_alone(hp, hp.train, reps)
     nums["alone_prefill"] = time_alone(hp, hp.prefill, reps)
     for i in range(len(hp.dec)):
