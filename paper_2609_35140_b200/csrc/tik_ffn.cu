@@ -83,22 +83,40 @@ __global__ void __launch_bounds__(HN_THREADS) rmsnorm_kernel(const NormParams p)
     }
 }
 
-// out[t][i] = silu(gu[t][i]) * gu[t][I + i]; one thread per 8 output elements.
+// out[t][i] = silu(gu[t][i]) * gu[t][I + i]; 16-byte vectors of 8 outputs, SW_VPT per thread (a block
+// covers 256 * SW_VPT consecutive vectors).  Large calls take four: all eight loads of a thread are
+// issued before the arithmetic, 128 bytes per thread in flight (6.3 -> 6.9 TB/s on 32 768 x 27 648);
+// small calls (decode) take one, which spreads them over more blocks.
+template <int SW_VPT>
 __global__ void __launch_bounds__(256) swiglu_kernel(const __nv_bfloat16* __restrict__ gu,
                                                     __nv_bfloat16* __restrict__ out, long long T, int I) {
     const int vpr = I / 8;                                   // output vectors per row
-    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (idx >= T * vpr) return;
-    const long long t = idx / vpr;
-    const int c = static_cast<int>(idx % vpr);
-    const uint4* row = reinterpret_cast<const uint4*>(gu) + t * 2 * vpr;
-    const uint4 gv = row[c], uv = row[vpr + c];
-    float g[8], u[8], o[8];
-    unpack8(gv, g);
-    unpack8(uv, u);
+    const long long nvec = T * vpr;
+    const long long base = static_cast<long long>(blockIdx.x) * (256 * SW_VPT) + threadIdx.x;
+    uint4 gv[SW_VPT], uv[SW_VPT];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) o[e] = swiglu_value(g[e], u[e]);
-    reinterpret_cast<uint4*>(out)[idx] = pack8(o);
+    for (int j = 0; j < SW_VPT; ++j) {
+        const long long idx = base + 256 * j;
+        if (idx < nvec) {
+            const long long t = idx / vpr;
+            const int c = static_cast<int>(idx - t * vpr);
+            const uint4* row = reinterpret_cast<const uint4*>(gu) + t * 2 * vpr;
+            gv[j] = row[c];
+            uv[j] = row[vpr + c];
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < SW_VPT; ++j) {
+        const long long idx = base + 256 * j;
+        if (idx < nvec) {
+            float g[8], u[8], o[8];
+            unpack8(gv[j], g);
+            unpack8(uv[j], u);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o[e] = swiglu_value(g[e], u[e]);
+            reinterpret_cast<uint4*>(out)[idx] = pack8(o);
+        }
+    }
 }
 
 template <bool RESIDUAL>
@@ -120,8 +138,12 @@ cudaError_t launch_rmsnorm(const NormParams& p, cudaStream_t stream) {
 cudaError_t launch_swiglu(const void* gu, void* out, long long T, int I, cudaStream_t stream) {
     if (T <= 0) return cudaSuccess;
     const long long n = T * (I / 8);
-    swiglu_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(gu), static_cast<__nv_bfloat16*>(out), T, I);
+    if (n >= (1ll << 20))
+        swiglu_kernel<4><<<static_cast<unsigned>((n + 1023) / 1024), 256, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(gu), static_cast<__nv_bfloat16*>(out), T, I);
+    else
+        swiglu_kernel<1><<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(gu), static_cast<__nv_bfloat16*>(out), T, I);
     return cudaGetLastError();
 }
 
