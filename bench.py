@@ -164,7 +164,8 @@ class HotPath:
             self.dec.append({
                 "ctx": torch.tensor(lens, dtype=torch.int32, device=dev), "max": max(lens),
                 "q": self.q[rows].contiguous(), "o": torch.empty(w.S, w.Hq, w.d, dtype=torch.bfloat16, device=dev),
-                "bytes": self._decode_bytes(lens), "label": c or "full"})
+                "bytes": self._decode_bytes(lens), "logical_bytes": sum(lens) * w.Hkv * w.d * 2 * 2,
+                "label": c or "full"})
         need = max(tik.workspace_bytes(tik.OP_ATTN_DECODE, w.S, w.Hq, w.Hkv, w.d, d["max"]) for d in self.dec)
         self.dec_ws = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
         self.o = torch.empty_like(self.q)
@@ -285,6 +286,45 @@ def time_alone(hp: HotPath, fn, reps: int, warmup: int = 2):
     torch.cuda.synchronize()
     ts = sorted(a.elapsed_time(b) for a, b in evs[warmup:])
     return ts[len(ts) // 2]
+
+
+def time_decode_graph(hp: HotPath, i: int, nsteps: int = 20):
+    """One decode point as a CUDA graph of `nsteps` identical steps (each: L2 flush, decode, combine),
+    replayed three times; the time of a graph of `nsteps` flushes alone is taken off.  Returns ms per
+    step, or None with the reason when the calls cannot be captured."""
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):                 # everything the capture needs has run once
+            hp.flush.zero_()
+            hp.decode(i)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g_all, g_flush = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_all):
+            for _ in range(nsteps):
+                hp.flush.zero_()
+                hp.decode(i)
+        with torch.cuda.graph(g_flush):
+            for _ in range(nsteps):
+                hp.flush.zero_()
+        ts = []
+        for g in (g_all, g_flush):
+            best = None
+            for _ in range(4):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                g.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                t = e0.elapsed_time(e1)
+                best = t if best is None else min(best, t)
+            ts.append(best)
+        del g_all, g_flush
+        return max(ts[0] - ts[1], 0.0) / nsteps, None
+    except Exception as exc:     # capture is an extra: the eager numbers stand without it
+        torch.cuda.synchronize()
+        return None, "%s: %s" % (type(exc).__name__, str(exc)[:200])
 
 
 # ------------------------------------------------------------------------------------------ end to end
@@ -630,13 +670,19 @@ def measure_workload(tik, w, steps, warmup, rank, local_rank, headline: bool, wa
     nums["alone_prefill"] = time_alone(hp, hp.prefill, reps)
     for i in range(len(hp.dec)):
         nums["alone_decode%d" % i] = time_alone(hp, lambda i=i: hp.decode(i), reps)
+    graph_notes = []
+    for i in range(len(hp.dec)):
+        ms_g, why = time_decode_graph(hp, i)
+        nums["graph_decode%d" % i] = ms_g if ms_g is not None else -1.0
+        graph_notes.append(why)
     nb = min(w.S, 256)
     hid_b, tgt_b = hp.hidden[:nb].contiguous(), hp.target[:nb].contiguous()
     lp_b = torch.empty(nb, dtype=torch.float32, device="cuda")
     nums["logprob_decode_shaped"] = time_alone(
         hp, lambda: tik.tik_token_logprob(hid_b, hp.W, tgt_b, ws=hp.lp_ws, logprob=lp_b), reps)
     info = {"clocks": clk, "region_s": region_s, "launches_per_step": hp.launches_per_step,
-            "dec": [{"label": d["label"], "bytes": d["bytes"]} for d in hp.dec], "lp_rows": nb}
+            "dec": [{"label": d["label"], "bytes": d["bytes"], "logical_bytes": d["logical_bytes"],
+                     "graph_note": graph_notes[j]} for j, d in enumerate(hp.dec)], "lp_rows": nb}
     if want_replay:
         ms, nsteps, launches = time_replay(hp)
         nums["replay_total"] = ms
@@ -677,10 +723,18 @@ def report_workload(w, nums, info, peaks, world):
         g = d["bytes"] / (t * 1e-3) / 1e9
         ta = nums["alone_decode%d" % i]
         ga = d["bytes"] / (ta * 1e-3) / 1e9
+        tg = nums.get("graph_decode%d" % i, -1.0)
+        graph = ({"ms_per_step": tg, "gbs": d["bytes"] / (tg * 1e-3) / 1e9, "frac_hbm": d["bytes"] / (tg * 1e-3) / 1e9 / hbm,
+                  "note": "CUDA graph of 20 identical steps (L2 flush + decode + combine each), the same graph of "
+                          "flushes alone taken off"} if tg > 0 else {"ms_per_step": None, "note": d.get("graph_note")})
         out["decode"].append({"context": d["label"], "ms": t, "gbs": g, "frac_hbm": g / hbm,
                               "frac_nominal_hbm": g / NOMINAL["hbm_gbs"], "unique_kv_bytes": d["bytes"],
+                              "logical_kv_bytes": d["logical_bytes"],
+                              "gbs_logical": d["logical_bytes"] / (t * 1e-3) / 1e9,
                               "tok_per_s": w.S * world / (t * 1e-3),
-                              "alone": {"ms": ta, "gbs": ga, "frac_hbm": ga / hbm}})
+                              "alone": {"ms": ta, "gbs": ga, "frac_hbm": ga / hbm,
+                                        "gbs_logical": d["logical_bytes"] / (ta * 1e-3) / 1e9},
+                              "graph20": graph})
     wb = w.vocab * w.hidden * 2
     t = nums["logprob_decode_shaped"]
     out["logprob_decode_shaped"] = {"rows": info["lp_rows"], "ms": t, "weight_bytes": wb, "gbs": wb / (t * 1e-3) / 1e9,
