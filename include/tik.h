@@ -73,6 +73,11 @@ const char* tik_contract_id(void);
  * this exercises that table with stand-in ordinals.  Needs no GPU.  Returns 0 when it holds. */
 int tik_selftest_host(void);
 
+/* Number of kernels the library has launched in this process so far (all contexts, all streams;
+ * every launch site counts itself when it enqueues a kernel).  No paper counterpart: it lets a
+ * benchmark state how many kernels a timed region launched.  Host only, never fails. */
+unsigned long long tik_kernel_launches(void);
+
 /* Scratch bytes an operator needs.  rows_or_batch: decode batch B, log-prob rows T, or the number
  * of sequences S for train forward / prefill.  max_ctx: the host's bound on a context length
  * (decode, prefill) or sequence length (train forward).  H, V only for the log-prob op.  Returns 0

@@ -48,6 +48,8 @@ def load(build_if_missing: bool = False) -> ctypes.CDLL:
     lib.tik_last_error.argtypes = [vp]
     lib.tik_last_error.restype = c.c_char_p
     lib.tik_contract_id.restype = c.c_char_p
+    lib.tik_kernel_launches.restype = c.c_ulonglong
+    lib.tik_kernel_launches.argtypes = []
     lib.tik_workspace_bytes.argtypes = [i32, i64, i32, i32, i32, i64, i32, i32]
     lib.tik_workspace_bytes.restype = sz
     lib.tik_device_status.argtypes = [vp, vp, c.POINTER(i32)]
@@ -122,6 +124,11 @@ def _stream():
 def workspace_bytes(op: int, rows_or_batch: int = 0, Hq: int = 0, Hkv: int = 0, d: int = 0,
                     max_ctx: int = 0, H: int = 0, V: int = 0) -> int:
     return int(load().tik_workspace_bytes(op, rows_or_batch, Hq, Hkv, d, max_ctx, H, V))
+
+
+def kernel_launches() -> int:
+    """Kernels the library has launched in this process so far."""
+    return int(load().tik_kernel_launches())
 
 
 def device_status() -> int:

@@ -83,7 +83,14 @@ static tik_status check_heads(tik_ctx* ctx, int Hq, int Hkv, int d, float scale)
 
 using namespace tik;
 
+namespace tik {
+std::atomic<unsigned long long> g_kernel_launches{0};
+}
+
 extern "C" {
+
+unsigned long long tik_kernel_launches(void) { return tik::g_kernel_launches.load(std::memory_order_relaxed); }
+
 
 tik_status tik_create(tik_ctx** out, int device) {
     if (!out) return TIK_ERR_INVALID_ARG;

@@ -539,6 +539,7 @@ static cudaError_t launch_bwd_t(dim3 grid, const CUtensorMap& tmQ, const CUtenso
         });
         if (e != cudaSuccess) return e;
     }
+    count_launch();
     kern<<<grid, BWD_THREADS, BwdSmem<D, MODE>::ALLOC, stream>>>(tmQ, tmK, tmV, tmDO, p);
     return cudaGetLastError();
 }
@@ -547,6 +548,7 @@ cudaError_t launch_attn_bwd(int d, int max_tiles, int S, const CUtensorMap& tmQ,
                             const CUtensorMap& tmV, const CUtensorMap& tmDO, const BwdParams& p,
                             const void* o, const void* dout, long long n_vec, cudaStream_t stream) {
     const unsigned dgrid = static_cast<unsigned>((n_vec * 32 + 255) / 256);
+    count_launch();  // exactly one of the launches below runs
     if (d == 128)
         bwd_delta_kernel<128><<<dgrid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(o),
                                                          static_cast<const __nv_bfloat16*>(dout), p.delta, n_vec);

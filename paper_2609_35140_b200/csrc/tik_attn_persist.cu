@@ -943,6 +943,7 @@ static cudaError_t launch_persist_t(int ncta, const CUtensorMap& tmQ, const CUte
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kern, tmQ, tmK, tmV, p, plan);
 }
 
@@ -994,6 +995,7 @@ cudaError_t launch_attn_persist(int d, bool paged, int sm_count, int S, int X, c
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     cudaError_t e = cudaLaunchKernelEx(&cfg, attn_plan_kernel, p.cu_seqlens, paged ? p.ctx_lens : static_cast<const int32_t*>(nullptr),
                                        S, split ? 7 : X - 1, static_cast<int4*>(plan));
     if (e != cudaSuccess) return e;

@@ -405,6 +405,7 @@ static cudaError_t launch_decode2_t(dim3 grid, const CUtensorMap& tmQ, const CUt
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kern, tmQ, tmK, tmV, p);
 }
 

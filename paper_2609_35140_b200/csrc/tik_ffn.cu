@@ -123,6 +123,7 @@ template <bool RESIDUAL>
 static cudaError_t launch_rmsnorm_t(const NormParams& p, cudaStream_t stream) {
     const unsigned grid = static_cast<unsigned>(p.T);
     const int nv = (p.H / 8 + HN_THREADS - 1) / HN_THREADS;
+    count_launch();  // exactly one of the launches below runs
     if (nv <= 1) rmsnorm_kernel<1, RESIDUAL><<<grid, HN_THREADS, 0, stream>>>(p);
     else if (nv <= 2) rmsnorm_kernel<2, RESIDUAL><<<grid, HN_THREADS, 0, stream>>>(p);
     else if (nv <= 4) rmsnorm_kernel<4, RESIDUAL><<<grid, HN_THREADS, 0, stream>>>(p);
@@ -138,6 +139,7 @@ cudaError_t launch_rmsnorm(const NormParams& p, cudaStream_t stream) {
 cudaError_t launch_swiglu(const void* gu, void* out, long long T, int I, cudaStream_t stream) {
     if (T <= 0) return cudaSuccess;
     const long long n = T * (I / 8);
+    count_launch();  // exactly one of the launches below runs
     if (n >= (1ll << 20))
         swiglu_kernel<4><<<static_cast<unsigned>((n + 1023) / 1024), 256, 0, stream>>>(
             static_cast<const __nv_bfloat16*>(gu), static_cast<__nv_bfloat16*>(out), T, I);

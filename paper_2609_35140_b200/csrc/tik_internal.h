@@ -18,6 +18,12 @@ struct tik_ctx {
 
 namespace tik {
 
+// Kernel launches issued by the library in this process (every launch site counts itself): what
+// tik_kernel_launches() reports, so that a caller can state how many kernels a region launched.
+extern std::atomic<unsigned long long> g_kernel_launches;
+inline void count_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
+
+
 // Runs a per-device set-up step (typically cudaFuncSetAttribute, whose effect belongs to the
 // current device's context) once for every device that reaches it.  One flag per device ordinal;
 // a failed step is retried by the next call.  Two threads racing on a device's first call may

@@ -429,6 +429,7 @@ static cudaError_t launch_linear_unit(const CUtensorMap& tmA, const CUtensorMap&
     });
     if (e != cudaSuccess) return e;
     const int grid = p.nunit < p.sm_count ? p.nunit : p.sm_count;
+    count_launch();
     linear_unit_kernel<<<grid, lin::THREADS, linu::ALLOC, stream>>>(tmA, tmB, tmY, p);
     return cudaGetLastError();
 }
@@ -465,6 +466,7 @@ static cudaError_t launch_linear_t(const CUtensorMap& tmA, const CUtensorMap& tm
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
 }
 

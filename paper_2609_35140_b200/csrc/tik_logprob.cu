@@ -407,6 +407,7 @@ static cudaError_t launch_logprob_main(const CUtensorMap& tmA, const CUtensorMap
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p);
 }
 
@@ -425,6 +426,7 @@ cudaError_t launch_logprob(const CUtensorMap& tmA, const CUtensorMap& tmB, const
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();  // exactly one of the launches below runs
     if (p.unit_mode) return cudaLaunchKernelEx(&cfg, logprob_finish_tiles_kernel, p);
     return cudaLaunchKernelEx(&cfg, logprob_finish_kernel, p);
 }

@@ -186,6 +186,7 @@ __global__ void __launch_bounds__(PREP_WARPS * 32, PREP_MIN_CTAS) prep_kernel(co
 cudaError_t launch_prep(int d, const PrepParams& p, int64_t total_new, cudaStream_t stream) {
     if (total_new <= 0) return cudaSuccess;
     const unsigned grid = static_cast<unsigned>((total_new + PREP_WARPS - 1) / PREP_WARPS);
+    count_launch();  // exactly one of the launches below runs
     if (d == 128) prep_kernel<128><<<grid, PREP_WARPS * 32, 0, stream>>>(p);
     else prep_kernel<64><<<grid, PREP_WARPS * 32, 0, stream>>>(p);
     return cudaGetLastError();
