@@ -513,6 +513,8 @@ def time_bwd(hp: "HotPath", burst, reps: int = 3):
     o = tik.tik_attn_train_fwd(hp.q, hp.k, hp.v, hp.cu, max(w.seq_lens), w.softmax_scale, lse=lse)
     ws = torch.empty(max(16, tik.workspace_bytes(tik.OP_ATTN_TRAIN_BWD, hp.q.shape[0], w.Hq, w.Hkv, w.d)),
                      dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    time.sleep(ALONE_PAUSE_S)
     ms = time_alone(hp, lambda: tik.tik_attn_train_bwd(hp.q, hp.k, hp.v, o, do, lse, hp.cu, max(w.seq_lens),
                                                         w.softmax_scale, ws=ws), reps, warmup=1)
     tf = 2.5 * w.train_flops() / (ms * 1e-3) / 1e12
@@ -875,8 +877,8 @@ def main():
             "bound": "hbm", "achieved": g, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": g / peaks["hbm_gbs"],
             "ms": t_prep, "bytes": b_prep,
             "note": "pre-attention step over all tokens of the workload; measured after the timed steps, not part of the metric"}
-        rooflines.update(time_ffn(hp, peaks, burst))    # timed alone: held against the burst peak
         rooflines["attn_train_bwd"] = time_bwd(hp, burst)
+        rooflines.update(time_ffn(hp, peaks, burst))    # timed alone: held against the burst peak
         flags |= tik.device_status()
 
     cpu = None
