@@ -65,7 +65,7 @@ def test_fused_residual_rmsnorm(tik, H):
     assert count_diff(y1, y[3:4]) == 0 and count_diff(r1, res[3:4]) == 0
 
 
-@pytest.mark.parametrize("T,I", [(1, 8), (33, 1000), (257, 8960), (64, 18944)])
+@pytest.mark.parametrize("T,I", [(1, 8), (33, 1000), (257, 8960), (64, 18944), (1100, 8960)])   # the last one: four vectors per thread, ragged last block
 def test_swiglu(tik, T, I):
     gu = _randn((T, 2 * I), 1000 + I, 3.0)
     gu[0, :4] = torch.tensor([0.0, 40.0, -40.0, -100.0], dtype=torch.bfloat16)
