@@ -201,6 +201,9 @@ tik_status tik_attn_prefill_kv(tik_ctx* ctx, const void* q, const void* k_new, c
  * ctx_lens[b] <= 0 is skipped and its output rows are left untouched.  The KV range is
  * split into fixed 2048-key chunks whose partial results go through `ws` and are folded in
  * ascending order by a second kernel on the same stream (fixed-order split-KV combine).
+ * With max_ctx_len <= 2048 every slot has one chunk, whose state is the result: the decode
+ * kernel then normalises and stores the rows itself (same operations, same bits), `ws` is
+ * not touched and no second kernel runs.
  * max_ctx_len is a host upper bound on ctx_lens[]: it sizes the grid and the scratch.  A slot
  * whose ctx_lens[b] exceeds it is computed over keys 0..max_ctx_len-1 only and raises
  * TIK_DEV_BAD_CONTEXT; nothing is written outside that slot's own scratch and output rows. */
