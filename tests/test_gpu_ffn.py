@@ -100,7 +100,7 @@ def test_linear_matches_oracle_and_is_batch_invariant(tik, T, K, N):
 @pytest.mark.parametrize("K,N", [(512, 37888), (256, 55296), (1024, 5120), (192, 1000), (128, 72), (64, 40000),
                                  (27648, 5120), (3584, 37888)])
 def test_decode_shaped_linear_equals_rows_of_a_batched_call(tik, K, N):
-    """One row tile (T <= 128) takes the persistent column-unit schedule with 128 or 256 columns
+    """One row tile (T <= 128) takes the persistent column-unit schedule with 64, 128 or 256 columns
     per unit and 32, 64 or 128 staged rows; every such call returns the bits of the same rows inside a
     300-row call (CTA pairs, 256-column steps), and writes nothing outside its [T][N] block.  Two row
     tiles (T <= 256) run the pair kernel persistently over 256-column steps: same check."""
