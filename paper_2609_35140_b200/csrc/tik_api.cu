@@ -415,15 +415,17 @@ tik_status tik_attn_decode(tik_ctx* ctx, const void* q, void* o, float* lse, con
     p.part_o = static_cast<float*>(ws);
     p.part_ml = p.part_o + static_cast<size_t>(B) * Hq * nchunk * d;
     p.dev_status = ctx->dev_status;
-    // Two kernels give the same bits.  The small CTA of tik_decode.cu (two per SM, every chunk
-    // resident at once) wins in the middle range: at most one (sequence, KV head) pair per SM but
-    // about as many chunks as SMs or more, where the one-CTA-per-SM kernel runs a ragged second wave.
-    // With fewer chunks than SMs every CTA has an SM to itself either way and that kernel's faster
-    // per-CTA pipeline (two softmax warpgroups, five K/V stages) gives the shorter latency; with
-    // more pairs than SMs the same pipeline streams faster per SM (measured on B200 at full and at
-    // power-capped clocks; the paper's decode grid, Sec. 6 Q3, covers both ends).
+    // Two kernels give the same bits.  The small CTA of tik_decode.cu (two per SM) wins where CTAs
+    // are short or few per SM: at most one (sequence, KV head) pair per SM but about as many chunks
+    // as SMs or more (the one-CTA-per-SM kernel runs a ragged second wave there), and any number of
+    // pairs with contexts of at most two chunks (a CTA streams <= 32 tiles; two co-resident CTAs hide
+    // each other's set-up and tail: 64 x 4096 keys 103 -> 93 us, 256 x 2048 395 -> 313 us, also
+    // right after a seconds-long GEMM).  With fewer chunks than SMs every CTA has an SM to itself
+    // either way and the big kernel's faster per-CTA pipeline (two softmax warpgroups, five K/V
+    // stages) gives the shorter latency; with many pairs of long contexts the same pipeline streams
+    // faster per SM (the paper's decode grid, Sec. 6 Q3, covers both ends).
     const long long pairs = static_cast<long long>(B) * Hkv;
-    const bool small_group = G <= DECODE2_MAX_G && pairs <= ctx->sm_count && 4 * pairs * nchunk >= 3ll * ctx->sm_count;
+    const bool small_group = G <= DECODE2_MAX_G && (pairs <= ctx->sm_count || nchunk <= 2) && 4 * pairs * nchunk >= 3ll * ctx->sm_count;
     p.cpc = decode_chunks_per_cta(B, Hkv, nchunk, ctx->sm_count, small_group ? 2 : 1);
     p.lookahead = ctx->sm_count;
     dim3 grid((nchunk + p.cpc - 1) / p.cpc, Hkv, B);

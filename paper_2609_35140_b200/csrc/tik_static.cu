@@ -146,7 +146,7 @@ extern "C" tik_status tik_attn_decode_static(const void* q, void* o, float* lse,
     if (!dev_flags) e = cudaMemsetAsync(s->flags, 0, sizeof(int), st);
     p.cpc = 1;
     if (e == cudaSuccess)
-        e = (G <= DECODE2_MAX_G && B * Hkv <= s->sm_count && 4ll * B * Hkv * nchunk >= 3ll * s->sm_count) ? launch_decode2(d, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st)
+        e = (G <= DECODE2_MAX_G && (B * Hkv <= s->sm_count || nchunk <= 2) && 4ll * B * Hkv * nchunk >= 3ll * s->sm_count) ? launch_decode2(d, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st)
                                : launch_attn(d, 2, dim3(nchunk, Hkv, B), tmQ, tmK, tmV, p, st);
     if (e == cudaSuccess && !p.direct_out) e = launch_combine(d, p, B, st);
     return e == cudaSuccess ? TIK_OK : TIK_ERR_CUDA;

@@ -59,3 +59,33 @@ def test_small_cta_decode_equals_train_rows(tik, G, Hkv, d, page, S):
                              torch.tensor([lens[s]], dtype=torch.int32, device="cuda"), kc, vc, bt[s][None].contiguous(),
                              lens[s], w.softmax_scale)
     assert count_diff(o1[0], o_train[int(cu_h[s]) + lens[s] - 1]) == 0
+
+
+@pytest.mark.parametrize("S,Hkv,G,lo,hi", [(150, 8, 2, 2049, 4096),     # 1200 pairs x 2 chunks: one CTA walks both chunks
+                                           (160, 4, 4, 1, 2048),        # 640 pairs x 1 chunk: the kernel finishes its rows itself
+                                           (40, 8, 1, 2049, 4000)])     # 320 pairs x 2 chunks, one chunk per CTA
+def test_small_cta_decode_with_more_pairs_than_sms(tik, S, Hkv, G, lo, hi):
+    """Contexts of at most two chunks take the small-CTA kernel whatever the number of (sequence,
+    KV head) pairs; the rows equal the packed train-forward's rows bit for bit."""
+    d, page = 128, 64
+    lens = _lens(7 * S + G, S, lo, hi)
+    lens[0], lens[1] = lo, hi
+    w = synth.custom_workload([1] * S, [L - 1 for L in lens], G * Hkv, Hkv, d, page)
+    q, k, v, cu = synth.make_qkv(w, "cuda")
+    o_train = tik.tik_attn_train_fwd(q, k, v, cu, max(lens), w.softmax_scale)
+    layout = synth.make_paged_layout(w)
+    bt = torch.from_numpy(layout.block_table).cuda()
+    kc = torch.zeros((layout.num_pages, Hkv, page, d), dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    ctx = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    tik.tik_kv_cache_write(k, v, cu, ctx, kc, vc, bt)
+    cu_h = w.cu_seqlens()
+    rows = torch.tensor([int(cu_h[s]) + lens[s] - 1 for s in range(S)], device="cuda")
+    lse = torch.zeros(S, w.Hq, dtype=torch.float32, device="cuda")
+    lse_train = torch.zeros(q.shape[0], w.Hq, dtype=torch.float32, device="cuda")
+    tik.tik_attn_train_fwd(q, k, v, cu, max(lens), w.softmax_scale, lse=lse_train)
+    n0 = tik.kernel_launches()
+    o = tik.tik_attn_decode(q[rows].contiguous(), ctx, kc, vc, bt, max(lens), w.softmax_scale, lse=lse)
+    assert tik.kernel_launches() - n0 == (1 if max(lens) <= 2048 else 2)
+    assert count_diff(o, o_train[rows]) == 0
+    assert count_diff(lse, lse_train[rows]) == 0
