@@ -612,14 +612,19 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     p.T = T;
     p.K = K;
     p.N = N;
-    // Columns per CTA: up to 4096 amortise a CTA's set-up and its last epilogue, which runs after
-    // the MMAs have ended; with few row tiles (decode) that would leave SMs idle, so the
-    // super-chunk shrinks until the grid covers the SMs four times.  An output element is one
-    // 256-column accumulator's chain over K either way: its bits do not depend on this choice.
+    // Columns per CTA (a "super-chunk" of 256-column steps): up to 16 steps amortise a CTA's set-up
+    // and its last epilogue, which runs after the MMAs have ended; with few row tiles that would leave
+    // SMs idle, so the number of super-chunks doubles until the grid covers the SMs four times.  The
+    // steps are then dealt evenly (N = 5120: two super-chunks of 10 steps, not 16 + 4, whose short
+    // CTAs left a quarter of the last wave idle).  An output element is one 256-column accumulator's
+    // chain over K either way: its bits do not depend on this choice.
     const long long ntile = (T + 127) / 128;
-    p.super_cols = 4096;
-    while (p.super_cols > 256 && ntile * ((N + p.super_cols - 1) / p.super_cols) < 4ll * ctx->sm_count) p.super_cols /= 2;
-    p.nsuper = (N + p.super_cols - 1) / p.super_cols;
+    const int steps = (N + 255) / 256;
+    int nsup = (steps + 15) / 16;
+    while (nsup < steps && ntile * nsup < 4ll * ctx->sm_count) nsup = nsup * 2 < steps ? nsup * 2 : steps;
+    const int per = (steps + nsup - 1) / nsup;
+    p.super_cols = per * 256;
+    p.nsuper = (steps + per - 1) / per;
     // two row tiles: the pair kernel, persistent over 256-column steps (decode batches up to 256)
     const bool pair_units = pair && T <= 256;
     p.unit_mode = (unit_mode || pair_units) ? 1 : 0;

@@ -177,7 +177,7 @@ struct LinearParams {
     __nv_bfloat16* y;            // [T][N]
     int64_t T;
     int K, N, nsuper;
-    int super_cols;              // output columns per CTA: 256 .. 4096 (a power of two)
+    int super_cols;              // output columns per CTA: a multiple of 256, at most 4096
     int unit_mode;               // T <= 128: persistent CTAs over column units (tmA box a_rows, tmB box nu rows)
     int nu, nunit, a_rows;       // unit width 64 / 128 / 256, ceil(N / nu), staged x rows 32 / 64 / 128
     int sm_count;
