@@ -625,11 +625,14 @@ tik_status tik_linear(tik_ctx* ctx, const void* x, const void* weight, void* y, 
     const int per = (steps + nsup - 1) / nsup;
     p.super_cols = per * 256;
     p.nsuper = (steps + per - 1) / per;
-    // two row tiles: the pair kernel, persistent over 256-column steps (decode batches up to 256)
-    const bool pair_units = pair && T <= 256;
+    // two to sixteen row tiles (decode batches up to 256, prefill-sized calls up to 2048 rows): the pair
+    // kernel, persistent over (256-column step, pair of row tiles) units -- a grid of one CTA pair per
+    // unit spends as long on set-up as on a unit's 56 .. 432 K slices, and x fits L2
+    const bool pair_units = pair && ntile <= 16;
     p.unit_mode = (unit_mode || pair_units) ? 1 : 0;
     p.nu = nu;
-    p.nunit = unit_mode ? (N + nu - 1) / nu : pair_units ? (N + 255) / 256 : 0;
+    p.ntp = static_cast<int>((ntile + 1) / 2);
+    p.nunit = unit_mode ? (N + nu - 1) / nu : pair_units ? steps * p.ntp : 0;
     p.a_rows = a_rows;
     p.sm_count = ctx->sm_count;
     p.dev_status = ctx->dev_status;

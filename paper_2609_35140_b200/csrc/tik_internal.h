@@ -179,6 +179,7 @@ struct LinearParams {
     int K, N, nsuper;
     int super_cols;              // output columns per CTA: a multiple of 256, at most 4096
     int unit_mode;               // T <= 128: persistent CTAs over column units (tmA box a_rows, tmB box nu rows)
+    int ntp;                     // pair unit mode: pairs of row tiles (1 .. 8)
     int nu, nunit, a_rows;       // unit width 64 / 128 / 256, ceil(N / nu), staged x rows 32 / 64 / 128
     int sm_count;
     int* dev_status;

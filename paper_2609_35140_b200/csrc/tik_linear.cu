@@ -55,14 +55,20 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const long long rem = blockIdx.x - band * per_band;
     const int sup = static_cast<int>(rem / BAND);
     const int tile_in_band = static_cast<int>(rem % BAND);
-    // unit mode (two row tiles, CTA pairs only): one persistent pair per two SMs walks the
-    // 256-column steps u = pair index, + number of pairs, ...; same MMA chain per element
+    // unit mode (up to 16 row tiles, CTA pairs only): one persistent pair per two SMs walks the
+    // units q = pair index, + number of pairs, ...; unit q = (256-column step q / ntp, pair of row
+    // tiles q % ntp): the pairs running at one time share a few steps of W in L2, and x (at most
+    // 2048 rows) stays there throughout.  Same MMA chain per element.
     const bool unit_mode = PAIR && p.unit_mode != 0;
     const int u_first = static_cast<int>(blockIdx.x >> 1), u_stride = static_cast<int>(gridDim.x >> 1);
     if (!unit_mode && (PAIR ? (tile_in_band & ~1) : tile_in_band) >= band_tiles) return;   // a pair leaves only together
-    const int row0 = unit_mode ? 128 * static_cast<int>(rank) : (band * BAND + tile_in_band) * 128;
-    const int col_base = unit_mode ? u_first * NB : sup * p.super_cols;
-    const int col_step = unit_mode ? u_stride * NB : NB;
+    const int row_fixed = (band * BAND + tile_in_band) * 128;
+    const int col_base = sup * p.super_cols;
+    const int ntp = unit_mode ? p.ntp : 1;
+    auto row_of = [&](int nt) {
+        return unit_mode ? (2 * ((u_first + nt * u_stride) % ntp) + static_cast<int>(rank)) * 128 : row_fixed;
+    };
+    auto col_of = [&](int nt) { return unit_mode ? ((u_first + nt * u_stride) / ntp) * NB : col_base + nt * NB; };
     const int n_nt = unit_mode ? (p.nunit - u_first + u_stride - 1) / u_stride
                                : min(p.super_cols / NB, (p.N - col_base + NB - 1) / NB);   // 256-column steps
     const int n_kb = p.K / 64;
@@ -118,7 +124,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         if (lane == 0) {
             uint32_t it = 0;
             for (int nt = 0; nt < n_nt; ++nt) {
-                const int col0 = col_base + nt * col_step;
+                const int col0 = col_of(nt), row0 = row_of(nt);
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
                     const int s = it % STAGES;
@@ -186,7 +192,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             const int buf = nt & 1;
             mbar_wait(bar_acc_full + 8 * buf, (nt >> 1) & 1, abort_word, p.dev_status);
             tc_fence_after();
-            const int col0 = col_base + nt * col_step;
+            const int col0 = col_of(nt), row0 = row_of(nt);
             const uint32_t taddr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * NB;
 #pragma unroll 1
             for (int q = 0; q < NB / 64; ++q, ++piece) {
