@@ -531,7 +531,8 @@ tik_status tik_token_logprob(tik_ctx* ctx, const void* hidden, const void* lm_he
         while (p.spc < 8 && ntile * ((p.nsuper + 2 * p.spc - 1) / (2 * p.spc)) >= 4ll * ctx->sm_count) p.spc *= 2;
     }
     p.unit_mode = T <= LP_UNIT_MODE_ROWS ? 1 : 0;
-    p.nunit = (V + 255) / 256;
+    p.ntp = pair ? static_cast<int>((T + 255) / 256) : 1;
+    p.nunit = ((V + 255) / 256) * p.ntp;
     p.ntile128 = (V + LP_TILE - 1) / LP_TILE;
     p.sm_count = ctx->sm_count;
     p.part_ml = static_cast<float*>(ws);

@@ -39,7 +39,7 @@ constexpr float LOG2E_F = 1.44269504088896340736f;
 constexpr float LN2_F = 0.69314718055994530942f;
 constexpr int LP_TILE = 128;          // vocabulary columns per log-sum-exp tile
 constexpr int LP_SUPER = 1024;        // vocabulary columns per super-chunk (8 tiles)
-constexpr int LP_UNIT_MODE_ROWS = 256; // log-prob calls of at most this many rows keep one partial per tile (schedule only)
+constexpr int LP_UNIT_MODE_ROWS = 2048; // log-prob calls of at most this many rows keep one partial per tile (schedule only)
 
 #define TIK_CONTRACT_ID "tik3-BN128-CH2048-M128N128K16-ex2ftz-lazy8-sum2x4-LP128x1024"
 

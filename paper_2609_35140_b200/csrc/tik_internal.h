@@ -152,8 +152,9 @@ struct LogprobParams {
     int64_t T;
     int H, V, nsuper;
     int spc;                     // consecutive 1024-column super-chunks walked by one CTA
-    int unit_mode;               // 1: T <= 256: persistent CTAs over 256-column steps, one (max, sum) pair per 128-column tile
-    int nunit, ntile128;         // ceil(V / 256), ceil(V / 128)
+    int unit_mode;               // 1: T <= LP_UNIT_MODE_ROWS: persistent CTAs over 256-column steps, one (max, sum) pair per 128-column tile
+    int nunit, ntile128;         // units = ceil(V / 256) x ntp, ceil(V / 128)
+    int ntp;                     // unit mode: pairs of token tiles (single CTAs: 1)
     int sm_count;
     float inv_temperature;
     int* dev_status;

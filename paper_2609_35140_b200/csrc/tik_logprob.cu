@@ -70,12 +70,21 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // accumulator steps u, u + n, u + 2n, ... of the vocabulary; every 128-column tile leaves its own
     // (max, sum) pair and the finish kernel folds them in the fixed order (tiles ascending inside a
     // super-chunk, then super-chunks ascending): the same operations on the same numbers.
+    // With more than two token tiles (up to LP_UNIT_MODE_ROWS rows) a unit is (256-column step,
+    // pair of token tiles), the pair index running fastest: the CTA pairs at work at one time share a
+    // few steps of lm_head in L2, and the hidden rows stay there throughout.
     const bool unit_mode = p.unit_mode != 0;
     const int u_first = static_cast<int>(blockIdx.x) / (PAIR ? 2 : 1);
     const int u_stride = static_cast<int>(gridDim.x) / (PAIR ? 2 : 1);
     const int n_my_units = unit_mode ? (u_first < p.nunit ? (p.nunit - 1 - u_first) / u_stride + 1 : 0) : 0;
     if (!unit_mode && (PAIR ? (tile_in_band & ~1) : tile_in_band) >= band_tiles) return;
-    const int tok0 = unit_mode ? (PAIR ? 128 * static_cast<int>(rank) : 0) : (band * BAND + tile_in_band) * 128;
+    const int ntp = unit_mode ? p.ntp : 1;
+    const int tok_fixed = (band * BAND + tile_in_band) * 128;
+    auto unit_col = [&](int sp) { return ((u_first + sp * u_stride) / ntp) * NB; };
+    auto unit_tok = [&](int sp) {
+        const int pi = (u_first + sp * u_stride) % ntp;
+        return (PAIR ? 2 * pi + static_cast<int>(rank) : pi) * 128;
+    };
     // 256-column accumulator steps of super-chunk sup0 + sp
     auto n_nt_of = [&](int sp) { return min(LP_SUPER / NB, (p.V - (sup0 + sp) * LP_SUPER + NB - 1) / NB); };
     const int n_kb = p.H / 64;
@@ -134,7 +143,8 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int n_sp_loop = unit_mode ? n_my_units : n_sp;
             for (int sp = 0; sp < n_sp_loop; ++sp)
             for (int nt = 0; nt < (unit_mode ? 1 : n_nt_of(sp)); ++nt) {
-                const int col0 = unit_mode ? (u_first + sp * u_stride) * NB : (sup0 + sp) * LP_SUPER + nt * NB;
+                const int col0 = unit_mode ? unit_col(sp) : (sup0 + sp) * LP_SUPER + nt * NB;
+                const int tok0 = unit_mode ? unit_tok(sp) : tok_fixed;
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     if (*abort_word) break;      // a wait expired somewhere: stop issuing copies
                     const int s = it % STAGES;
@@ -195,14 +205,19 @@ logprob_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
         const int row = quarter * 32 + lane;
-        const long long t = static_cast<long long>(tok0) + row;
-        const bool row_valid = t < p.T;
-        const int target = row_valid ? p.target[t] : -1;
+        long long t = static_cast<long long>(tok_fixed) + row;
+        bool row_valid = t < p.T;
+        int target = (!unit_mode && row_valid) ? p.target[t] : -1;
         const float it_scale = p.inv_temperature;
         uint32_t acc = 0;
         const int n_sp_loop = unit_mode ? n_my_units : n_sp;
         for (int sp = 0; sp < n_sp_loop; ++sp) {
-        const int col_base = unit_mode ? (u_first + sp * u_stride) * NB : (sup0 + sp) * LP_SUPER;
+        const int col_base = unit_mode ? unit_col(sp) : (sup0 + sp) * LP_SUPER;
+        if (unit_mode) {                                   // the unit's token tile
+            t = static_cast<long long>(unit_tok(sp)) + row;
+            row_valid = t < p.T;
+            target = row_valid ? p.target[t] : -1;
+        }
         float M = -CUDART_INF_F, Lsum = 0.0f;
         bool first = true;
         for (int nt = 0; nt < (unit_mode ? 1 : n_nt_of(sp)); ++nt, ++acc) {

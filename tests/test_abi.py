@@ -37,9 +37,11 @@ def test_host_only_calls_work_without_a_gpu():
     # decode scratch: B * Hq * chunks * (d + 4) floats; log-prob: T * (2 * super-chunks + 1) floats
     assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 16384) == 16 * 32 * 8 * 132 * 4
     assert binding.workspace_bytes(binding.OP_ATTN_DECODE, 16, 32, 8, 128, 2049) == 16 * 32 * 2 * 132 * 4
-    assert binding.workspace_bytes(binding.OP_TOKEN_LOGPROB, 1000, H=4096, V=151936) == 1000 * (2 * 149 + 1) * 4
-    # decode-sized calls (<= 256 rows) keep one partial per 128-column tile: ceil(151936 / 128) = 1187
+    assert binding.workspace_bytes(binding.OP_TOKEN_LOGPROB, 5000, H=4096, V=151936) == 5000 * (2 * 149 + 1) * 4
+    # calls of at most 2048 rows keep one partial per 128-column tile: ceil(151936 / 128) = 1187
     assert binding.workspace_bytes(binding.OP_TOKEN_LOGPROB, 64, H=4096, V=151936) == 64 * (2 * 1187 + 1) * 4
+    assert binding.workspace_bytes(binding.OP_TOKEN_LOGPROB, 2048, H=4096, V=151936) == 2048 * (2 * 1187 + 1) * 4
+    assert binding.workspace_bytes(binding.OP_TOKEN_LOGPROB, 2049, H=4096, V=151936) == 2049 * (2 * 149 + 1) * 4
     # full-sequence kernels: a plan of 16 bytes per (sequence, candidate item) + header; 4096 positions
     # = 32 tiles = 8 pairs + 16 single tiles
     assert binding.workspace_bytes(binding.OP_ATTN_TRAIN_FWD, 1000, 8, 2, 128, 4096) == 16 + 16 * 1000 * 24

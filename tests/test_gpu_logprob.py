@@ -80,6 +80,22 @@ def test_batch_shape_invariance(tik):
         assert count_diff(full[a:b], part) == 0, (a, b)
 
 
+def test_mid_sized_calls_equal_rows_of_a_large_call(tik):
+    """Calls of 3 to 16 token tiles run persistently over (vocabulary step, pair of token tiles)
+    units with one partial per 128-column tile; a larger call keeps one partial per 1024 columns.
+    Same rows, same bits; sampled rows against the oracle."""
+    T, H, V = 2500, 192, 5000 + 8
+    hidden, W, target = _inputs(T, H, V, 99, 0.3)
+    target[:3] = torch.tensor([0, V - 1, 4095], dtype=torch.int32)
+    full = tik.tik_token_logprob(hidden, W, target)
+    rows = torch.tensor([0, 1, 2, 255, 256, 257, 1023, 1024, 2047, 2048, T - 1], device="cuda")
+    ref, _ = _oracle(hidden[rows], W, target[rows])
+    assert np.abs(full[rows].cpu().numpy() - ref).max() <= LOGPROB_TOL
+    for a, b in [(0, 700), (300, 2348), (1000, 1513), (2100, 2500), (0, 257), (1, 2049)]:
+        part = tik.tik_token_logprob(hidden[a:b].contiguous(), W, target[a:b].contiguous())
+        assert count_diff(full[a:b], part) == 0, (a, b)
+
+
 def test_two_bands_several_super_chunks_per_cta(tik):
     """More than one band of 32 token tiles (the second one a single, partner-less tile) and enough
     work that a CTA walks two super-chunks: sampled rows against the oracle, slices bit for bit."""
