@@ -1017,37 +1017,72 @@ __global__ void __launch_bounds__(D) combine_kernel(const AttnParams p) {
 }
 
 // ------------------------------------------------------------------ KV-cache write
-__global__ void __launch_bounds__(128)
+// A block copies KVW_TOK (8 or 1) consecutive new tokens (K and V rows of all KV heads: 16-byte vectors).
+// Threads 0 .. KVW_TOK-1 find their token's sequence (binary search over cu_new), position and
+// physical page; then all threads copy, every thread's loads issued before its stores.  (One token
+// per 128-thread block, each doing its own search before 32 bytes of copying per thread, reached
+// 0.76 of the copy bandwidth.)
+constexpr int KVW_THREADS = 256;
+template <int KVW_TOK>       // 8 for prompts, 1 for a decode step's handful of tokens (more blocks, shorter chains)
+__global__ void __launch_bounds__(KVW_THREADS)
 kv_write_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                 const int32_t* __restrict__ cu_new, const int32_t* __restrict__ ctx_lens,
                 uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
-                const int32_t* __restrict__ block_table, int max_blocks, int S, int Hkv,
+                const int32_t* __restrict__ block_table, int max_blocks, int S, long long total_new, int Hkv,
                 int vec_per_head /* d*2/16 */, int page_size, int num_pages, int* dev_status) {
     pdl_launch_dependents();       // an attention kernel launched next may be scheduled behind this grid
-    const int token = blockIdx.x;
-    int lo = 0, hi = S;            // find s with cu_new[s] <= token < cu_new[s+1]
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (cu_new[mid] <= token) lo = mid; else hi = mid;
+    __shared__ long long dst_base[KVW_TOK];     // vector index of (page, head 0, row, 0), or -1
+    const long long tok0 = static_cast<long long>(blockIdx.x) * KVW_TOK;
+    if (threadIdx.x < KVW_TOK) {
+        const long long token = tok0 + threadIdx.x;
+        long long base = -1;
+        if (token < total_new) {
+            int lo = 0, hi = S;            // find s with cu_new[s] <= token < cu_new[s+1]
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (cu_new[mid] <= token) lo = mid; else hi = mid;
+            }
+            const int s = lo;
+            const int n_s = cu_new[s + 1] - cu_new[s];
+            const int pos = ctx_lens[s] - n_s + static_cast<int>(token - cu_new[s]);
+            if (token < cu_new[s + 1] && pos >= 0) {
+                const int lp = pos / page_size, row = pos % page_size;
+                const int phys = (lp < max_blocks) ? block_table[static_cast<long long>(s) * max_blocks + lp] : -1;
+                if (phys < 0 || phys >= num_pages) atomicOr(dev_status, TIK_DEV_BAD_BLOCK);
+                else base = (static_cast<long long>(phys) * Hkv * page_size + row) * vec_per_head;
+            }
+        }
+        dst_base[threadIdx.x] = base;
     }
-    const int s = lo;
-    const int n_s = cu_new[s + 1] - cu_new[s];
-    if (token >= cu_new[s + 1]) return;
-    const int pos = ctx_lens[s] - n_s + (token - cu_new[s]);
-    if (pos < 0) return;
-    const int lp = pos / page_size, row = pos % page_size;
-    int phys = (lp < max_blocks) ? block_table[static_cast<long long>(s) * max_blocks + lp] : -1;
-    if (phys < 0 || phys >= num_pages) {
-        if (threadIdx.x == 0) atomicOr(dev_status, TIK_DEV_BAD_BLOCK);
-        return;
-    }
-    const int nvec = Hkv * vec_per_head;
-    for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
-        const int hh = i / vec_per_head, e = i % vec_per_head;
-        const long long dst = ((static_cast<long long>(phys) * Hkv + hh) * page_size + row) * vec_per_head + e;
-        const long long src = static_cast<long long>(token) * nvec + i;
-        k_cache[dst] = k_new[src];
-        v_cache[dst] = v_new[src];
+    __syncthreads();
+    const int nvec = Hkv * vec_per_head;                 // vectors per token and tensor
+    const int per_block = KVW_TOK * nvec;
+    const long long head_pitch = static_cast<long long>(page_size) * vec_per_head;
+    for (int i0 = threadIdx.x; i0 < per_block; i0 += 4 * KVW_THREADS) {
+        uint4 kv[4], vv[4];
+        long long dst[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * KVW_THREADS;
+            dst[u] = -1;
+            if (i < per_block) {
+                const int j = i / nvec, r = i - j * nvec;          // token of the block, vector of the token
+                const long long base = dst_base[j];
+                if (base >= 0) {
+                    const int hh = r / vec_per_head, e = r - hh * vec_per_head;
+                    dst[u] = base + hh * head_pitch + e;
+                    const long long src = (tok0 + j) * nvec + r;
+                    kv[u] = k_new[src];
+                    vv[u] = v_new[src];
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (dst[u] >= 0) {
+                k_cache[dst[u]] = kv[u];
+                v_cache[dst[u]] = vv[u];
+            }
     }
 }
 
@@ -1112,11 +1147,17 @@ cudaError_t launch_kv_write(const void* k_new, const void* v_new, const int32_t*
                             int Hkv, int d, int page_size, int num_pages, int* dev_status,
                             cudaStream_t stream) {
     if (total_new <= 0) return cudaSuccess;
-    count_launch();
-    kv_write_kernel<<<static_cast<unsigned>(total_new), 128, 0, stream>>>(
-        static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), cu_new, ctx_lens,
-        static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), block_table, max_blocks, S, Hkv,
-        d * 2 / 16, page_size, num_pages, dev_status);
+    count_launch();  // exactly one of the launches below runs
+    if (total_new >= 4096)
+        kv_write_kernel<8><<<static_cast<unsigned>((total_new + 7) / 8), KVW_THREADS, 0, stream>>>(
+            static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), cu_new, ctx_lens,
+            static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), block_table, max_blocks, S, total_new, Hkv,
+            d * 2 / 16, page_size, num_pages, dev_status);
+    else
+        kv_write_kernel<1><<<static_cast<unsigned>(total_new), KVW_THREADS, 0, stream>>>(
+            static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), cu_new, ctx_lens,
+            static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), block_table, max_blocks, S, total_new, Hkv,
+            d * 2 / 16, page_size, num_pages, dev_status);
     return cudaGetLastError();
 }
 
